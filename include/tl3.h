@@ -1,0 +1,148 @@
+/*
+ * tl3 -- C ABI of the three-layer sparse-weight SpMM library for NVIDIA B200 (sm_100a).
+ *
+ * The library stores an fp16 weight matrix W (M x K, ~50 % unstructured sparsity) in the paper's
+ * three-layer format (Sec. 3.2: Sparse-TC layer, Slot-Filling layer with parallel-differential-
+ * distance position codes, Residual layer) and computes Y = W X for a small-N fp16 activation
+ * block X (Sec. 5.1: W is M x K, X is K x N, Y is M x N) with hand-written CUDA kernels that run
+ * the Sparse-TC layer on the sparse tensor cores and decode the other two layers on chip
+ * (Sec. 4).  The format is built once, ahead of time, on the host (Sec. 2.1).
+ *
+ * Conventions
+ *   - Every function returns TL3_OK (0) or a negative TL3_ERR_* code; nothing throws, exits or
+ *     synchronises the device unless stated.
+ *   - "host" / "device" in a comment says where the pointer must point.
+ *   - fp16 values cross the ABI as their 16-bit patterns (uint16_t).
+ *   - The handle owns its host copies of the format.  The caller owns ALL device memory (the
+ *     packed weight blob, X, Y, the workspace) and keeps it alive while work is queued.
+ *   - There is no CPU fallback: tl3_spmm fails if no sm_100 device is current.
+ */
+#ifndef TL3_H_
+#define TL3_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tl3_matrix tl3_matrix;          /* opaque */
+
+/* Tile of the format: pairing of surplus weights with empty slots and the 16-bit start
+ * positions of Algorithm 1 are local to one tile (Sec. 4.2 loads the matrix tile by tile).
+ * NULL means {128, 128, 15}; the GPU kernels accept only that default. */
+typedef struct {
+  int32_t tile_m;   /* rows per tile, > 0                                             */
+  int32_t tile_k;   /* columns per tile, multiple of 8, tile_m*tile_k/2 <= 65535      */
+  int32_t maxd;     /* largest 4-bit differential distance, 1..15 (0 marks a dummy)   */
+} tl3_params;
+
+/* Non-zero counts by layer (Sec. 3.2 quotes their shares) and sizes in bytes. */
+typedef struct {
+  int64_t M, K, M_pad, K_pad, n_tiles;
+  int64_t nnz, n_tc, n_sf, n_res, n_dummy, n_slots_unused;
+  int64_t canonical_bytes;    /* sum of the nine canonical arrays                     */
+  int64_t device_bytes;       /* size of the packed device blob                       */
+} tl3_stats_t;
+
+enum {
+  TL3_OK = 0,
+  TL3_ERR_INVALID_ARG = -1,
+  TL3_ERR_UNSUPPORTED = -2,      /* N, tile shape or device not supported by the kernels       */
+  TL3_ERR_NOT_UPLOADED = -3,
+  TL3_ERR_BAD_CONTAINER = -4,    /* inconsistent container (deserialize / decode)               */
+  TL3_ERR_CUDA = -5,             /* a CUDA runtime call failed; see tl3_last_cuda_error()       */
+  TL3_ERR_DEVICE_TIMEOUT = -6,   /* a bounded wait inside the kernel gave up (status word)      */
+  TL3_ERR_NO_MEMORY = -7
+};
+
+/* Canonical arrays, in the order tl3_canonical() numbers them. */
+enum {
+  TL3_TC_VALS = 0,     /* u16 [M_pad][K_pad/2]  two value slots per window of four weights      */
+  TL3_TC_META = 1,     /* u8  [M_pad][K_pad/8]  nibble idx0|idx1<<2 per window, even window low  */
+  TL3_CHAIN_TAU0 = 2,  /* u16 [tiles][tile_m]   first offset_t of each chain (Algorithm 1 l.3)   */
+  TL3_CHAIN_RHO0 = 3,  /* u16 [tiles][tile_m]   first offset_r of each chain (Algorithm 1 l.4)   */
+  TL3_CHAIN_LEN = 4,   /* u8  [tiles][tile_m]   number of delta bytes of each chain              */
+  TL3_PDD_BYTES = 5,   /* u8  []                t delta low nibble, r delta high nibble          */
+  TL3_TILE_DIR = 6,    /* u32 [tiles][4]        pdd_off, pdd_len, res_off, res_cnt               */
+  TL3_RES_RHO = 7,     /* u16 []                Residual positions                               */
+  TL3_RES_VAL = 8      /* u16 []                Residual values                                  */
+};
+
+/* ---- format: host side (Sec. 3.2) ------------------------------------------------------ */
+
+/* Encode a dense, already masked matrix (pruned weights are zeros; -0.0 counts as zero).
+ * W: host, fp16 bits, row-major M x K, leading dimension K.  *out receives a new handle that the
+ * caller releases with tl3_free().  Errors: INVALID_ARG (NULL, M or K <= 0, bad params). */
+int tl3_encode(const uint16_t* W, int64_t M, int64_t K, const tl3_params* params, tl3_matrix** out);
+
+/* Decode back to dense: Algorithm 1 run on the host, then the 2:4 expansion and the Residual
+ * entries.  W_out: host, M*K uint16_t, caller-owned, fully overwritten.  The result equals the
+ * encoder's input bit for bit (with -0.0 read as +0.0).  Errors: BAD_CONTAINER. */
+int tl3_decode(const tl3_matrix* m, uint16_t* W_out);
+
+/* Borrow one canonical array (TL3_TC_VALS ...).  *ptr stays valid until tl3_free(). */
+int tl3_canonical(const tl3_matrix* m, int which, const void** ptr, size_t* bytes);
+
+int tl3_stats(const tl3_matrix* m, tl3_stats_t* out);
+
+/* Bit-exact persistence of the canonical container ("stored ahead of time", Sec. 2.1).
+ * tl3_serialize: buf == NULL writes the needed size to *bytes; otherwise *bytes is the capacity
+ * on entry and the size written on return.  buf: host. */
+int tl3_serialize(const tl3_matrix* m, void* buf, size_t* bytes);
+int tl3_deserialize(const void* buf, size_t bytes, tl3_matrix** out);
+
+void tl3_free(tl3_matrix* m);
+
+/* ---- device side (Sec. 4) -------------------------------------------------------------- */
+
+/* Size of the packed device blob (tile blocks ready for bulk copies). */
+size_t tl3_device_bytes(const tl3_matrix* m);
+
+/* Pack the container and copy it to dptr (device, >= tl3_device_bytes(), 256-byte aligned) on
+ * `stream` (a cudaStream_t passed as void*; NULL = default stream), then bind dptr to the handle.
+ * The copy is asynchronous with respect to the device; host staging is released before return.
+ * Errors: UNSUPPORTED (tile shape other than 128 x 128), INVALID_ARG, CUDA. */
+int tl3_upload(tl3_matrix* m, void* dptr, void* stream);
+
+/* Scratch the kernel needs for N columns: split-K partial sums, arrival counters, a status word.
+ * Depends on the current device's SM count.  The caller allocates it (device, 256-byte aligned),
+ * clears it once with tl3_workspace_init(), and may then reuse it for any number of calls that
+ * do not overlap on the GPU (the kernel leaves it cleared). */
+size_t tl3_workspace_bytes(const tl3_matrix* m, int N);
+int tl3_workspace_init(void* workspace, size_t bytes, void* stream);
+
+/* Y = W X  (Sec. 5.1 problem statement; kernel design after Sec. 4: tile-wise streaming of the
+ * compressed weights, on-chip PDD decoding per Algorithm 1, sparse tensor-core MMA, Residual
+ * folded into the same accumulators, one final reduction).
+ *   X: device, fp16, K x N row-major, leading dimension ldx >= N, ldx % 8 == 0, 16-byte aligned.
+ *   Y: device, fp16, M x N row-major, leading dimension ldy >= N; fully overwritten.
+ *   1 <= N <= 64.  fp32 accumulation, fp16 round-to-nearest-even output.  W and X are assumed
+ *   finite (an empty slot multiplies an exact zero with an element of X).
+ * Asynchronous on `stream`; allocates nothing; does not synchronise.  Calls that share a
+ * workspace must not overlap on the GPU.
+ * Errors: NOT_UPLOADED, INVALID_ARG, UNSUPPORTED (N out of range, device is not sm_100), CUDA. */
+int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N,
+             void* workspace, void* stream);
+
+/* Same product with HOST buffers: copies X to dX, runs tl3_spmm, copies dY to Y and waits for the
+ * stream.  X, Y: host (pinned memory makes the copies asynchronous), dense leading dimensions
+ * ldx = ldy = N.  dX (>= K*N*2 bytes) and dY (>= M*N*2 bytes): device scratch owned by the caller. */
+int tl3_spmm_host(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int N, void* dX, void* dY,
+                  void* workspace, void* stream);
+
+/* Read the workspace's status word (synchronises `stream`).  TL3_OK, or DEVICE_TIMEOUT if a
+ * bounded wait inside a kernel expired since the last tl3_workspace_init(). */
+int tl3_status(const tl3_matrix* m, void* workspace, void* stream);
+
+/* Kernel launch geometry of the last tl3_spmm on this handle (for reporting): CTAs, stages. */
+int tl3_last_launch(const tl3_matrix* m, int* ctas, int* stages, int* smem_bytes);
+
+const char* tl3_strerror(int code);
+int tl3_last_cuda_error(void);      /* cudaError_t of the last failed runtime call, this thread */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TL3_H_ */

@@ -1,0 +1,71 @@
+// Internal definitions shared by the host-side and CUDA-side translation units of libtl3.
+#pragma once
+#include <cstdint>
+#include <cstddef>
+#include <vector>
+
+#include "tl3.h"
+
+struct tl3_matrix {
+  int64_t M = 0, K = 0, M_pad = 0, K_pad = 0;
+  int64_t tiles_m = 0, tiles_k = 0, n_tiles = 0;
+  tl3_params p{128, 128, 15};
+
+  // canonical container (Sec. 3.2)
+  std::vector<uint16_t> tc_vals;
+  std::vector<uint8_t> tc_meta;
+  std::vector<uint16_t> chain_tau0, chain_rho0;
+  std::vector<uint8_t> chain_len;
+  std::vector<uint8_t> pdd_bytes;
+  std::vector<uint32_t> tile_dir;      // 4 per tile: pdd_off, pdd_len, res_off, res_cnt
+  std::vector<uint16_t> res_rho, res_val;
+
+  // layer statistics
+  int64_t nnz = 0, n_tc = 0, n_sf = 0, n_res = 0, n_dummy = 0, n_slots_unused = 0;
+
+  // device binding (filled by tl3_upload)
+  void* dptr = nullptr;
+  size_t device_bytes = 0;             // computed lazily by tl3_device_bytes
+  uint32_t max_block_bytes = 0;
+  size_t dir_offset = 0, blocks_offset = 0;
+
+  // last launch geometry
+  mutable int last_ctas = 0, last_stages = 0, last_smem = 0;
+};
+
+namespace tl3 {
+
+// ---- device blob layout ------------------------------------------------------------------
+// [0, 256)                 header (magic, shape; informational)
+// [dir_offset, ...)        one DirEntry per tile
+// [blocks_offset, ...)     tile blocks, each 128-byte aligned, row-tile-major
+//
+// Tile block (tile 128 x 128, H = 64 value slots per row):
+//   +0      values   128 rows x 128 B, the K-major 128-byte-swizzled image the MMA descriptor
+//                    reads: 16-byte chunk j of row r sits at chunk (j ^ (r & 7))
+//   +16384  metadata 128 x 16 B: word kb of entry L is the TMEM word of lane L for k-block kb:
+//                    bits 0-15 = nibbles of windows 8kb+4h .. 8kb+4h+3 of row (L&7)+16(L>>4),
+//                    bits 16-31 = the same windows of that row + 8, with h = (L>>3)&1
+//   +18432  u32[4]: pdd_len, res_cnt, 0, 0
+//   +18448  chain starts u32[128]: tau0 | rho0 << 16 (0xFFFFFFFF = empty chain)
+//   +18960  chain lengths u8[128]
+//   +19088  PDD delta bytes, chain-major, padded to 4 bytes
+//   +...    Residual entries u32[res_cnt]: rho | value << 16, padded to 16 bytes
+constexpr int kTileM = 128, kTileK = 128, kH = 64;
+constexpr uint32_t kValsBytes = 16384, kMetaOff = 16384, kMetaBytes = 2048;
+constexpr uint32_t kInfoOff = 18432, kHdrOff = 18448, kLenOff = 18960, kPddOff = 19088;
+constexpr uint32_t kBlockAlign = 128;
+
+struct DirEntry {
+  uint32_t off16;     // block offset from the blob base, in 16-byte units
+  uint32_t bytes;     // block size (multiple of 16)
+  uint32_t pdd_len;
+  uint32_t res_cnt;
+};
+
+size_t plan_device_layout(tl3_matrix* m);                 // fills device_bytes, offsets, max block
+void pack_device_blob(const tl3_matrix* m, uint8_t* out); // out: device_bytes bytes, host
+
+void set_cuda_error(int e);
+
+}  // namespace tl3

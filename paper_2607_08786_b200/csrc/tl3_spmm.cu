@@ -1,0 +1,761 @@
+// Device side of libtl3: upload, workspace, and the SpMM kernel for sm_100a.
+//
+// Kernel design (what the paper's Sec. 4 pipeline becomes on B200):
+//   * one persistent CTA per SM owns a contiguous range of 128 x 128 tiles in row-tile-major
+//     order (split-K: a row-tile may be shared by several CTAs);
+//   * a producer warp streams each tile's packed block (values + metadata + PDD codes + Residual)
+//     with ONE bulk copy and the matching 128 x N block of X with one TMA tensor copy into a ring
+//     of shared-memory stages (Sec. 4.2 "Efficient Matrix Loading": W streamed tile by tile, X
+//     small enough to live in L2);
+//   * two groups of four decode warps alternate over the tiles: copy the 2-bit metadata to tensor
+//     memory, run Algorithm 1 (one PDD chain per thread; chain byte offsets by a warp-shuffle
+//     prefix sum of the chain lengths) moving each parked value from W_t to a second 2:4 operand
+//     W_r and zeroing its slot, and scatter the Residual entries into W_r as well
+//     (Sec. 4.3; surplus weights always sit at in-window index 2 or 3, so W_r's metadata is the
+//     constant pattern {2,3});
+//   * one thread issues tcgen05.mma.sp (kind::f16, M = 128, K = 32) on W_t and on W_r into the
+//     same fp32 accumulator in tensor memory (Sec. 4.3 "Sparse TC Computation");
+//   * four epilogue warps read the accumulator; a row-tile owned by one CTA is written to Y
+//     directly, otherwise partial sums go to the workspace and the last CTA to arrive adds them in
+//     a fixed order (Sec. 4.4: a single reduction at the end of the pipeline).
+// Every wait is bounded: on expiry the CTA records a code in the workspace status word, stops
+// issuing work, waits for its copies in flight, frees its tensor memory and returns.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+
+#include <cstdint>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "tl3_internal.h"
+
+namespace tl3 {
+
+static thread_local int g_last_cuda_error = 0;
+void set_cuda_error(int e) { g_last_cuda_error = e; }
+
+#define TL3_CUDA(expr)                                        \
+  do {                                                        \
+    cudaError_t e_ = (expr);                                  \
+    if (e_ != cudaSuccess) {                                  \
+      tl3::set_cuda_error(static_cast<int>(e_));              \
+      return TL3_ERR_CUDA;                                    \
+    }                                                         \
+  } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// Kernel configuration
+// ---------------------------------------------------------------------------------------------
+constexpr int kThreads = 512;             // 16 warps
+constexpr int kProducerWarp = 0;
+constexpr int kMmaWarp = 1;
+constexpr int kAllocWarp = 2;
+constexpr int kDecodeWarp0 = 4;           // warps 4-7: decode group 0, warps 8-11: group 1
+constexpr int kEpilogueWarp0 = 12;        // warps 12-15
+constexpr int kGroups = 2;
+constexpr int kMaxStages = 8;
+constexpr uint32_t kWrBytes = 16384;
+constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kColMetaT = 128;       // + 4 * group
+constexpr uint32_t kColMetaR = 136;       // two columns of 0xEEEEEEEE
+constexpr uint32_t kSmemLimit = 232448;   // 227 KB
+constexpr uint32_t kBarrierBytes = 1024;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per kernel
+
+// status codes written to the workspace status word (0 = ok)
+enum : uint32_t {
+  kStProducer = 1, kStDecodeFull = 2, kStDecodeWrFree = 3, kStMmaDecoded = 4, kStMmaAccEmpty = 5,
+  kStEpilogueAccFull = 6, kStDrain = 7
+};
+
+struct KernelArgs {
+  const uint8_t* blob;       // base of the packed blob (device)
+  const DirEntry* dir;       // tile directory (device)
+  long long total_tiles;
+  int tiles_m, tiles_k;
+  int M, N;
+  long long ldy;
+  __half* Y;
+  float* partials;           // [2 * gridDim.x][n_pad][128]
+  unsigned int* counters;    // [tiles_m]
+  unsigned int* status;      // status word
+  uint32_t stage_stride;     // bytes per stage (block area + X tile), multiple of 1024
+  uint32_t x_offset;         // offset of the X tile inside a stage, multiple of 1024
+  int num_stages;
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ unsigned long long global_timer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred q;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+  return done != 0;
+}
+
+// Shared state every wait looks at: the abort flag (set by whoever gives up first), the status
+// word in global memory and the kernel's start time.
+struct WaitCtx {
+  volatile int* abort_flag;
+  unsigned int* status;
+  unsigned long long t0;
+};
+
+// Bounded wait.  Returns false if the CTA is aborting (this or another waiter ran out of time).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w, uint32_t code) {
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 255u) {
+      if (*w.abort_flag) return false;
+      if (global_timer() - w.t0 > kWaitLimitNs) {
+        atomicCAS(w.status, 0u, code);
+        *w.abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// barrier + AND-reduction of a predicate over the `threads` threads that use barrier `id`
+__device__ __forceinline__ bool named_bar_all(int id, int threads, bool pred) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %3, 0;\n\t"
+      "bar.red.and.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(out) : "r"(id), "r"(threads), "r"(static_cast<uint32_t>(pred)) : "memory");
+  return out != 0;
+}
+
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void umma_sp_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t e_tmem,
+                                            uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// byte offset of value slot `pos` (row = pos / 64, slot = pos % 64) inside a 128 x 128-byte
+// K-major tile with the 128-byte swizzle: 16-byte chunk index ^= row & 7
+__device__ __forceinline__ uint32_t swizzled_offset(uint32_t pos) { return (pos << 1) ^ ((pos >> 2) & 0x70u); }
+
+template <int NPAD> struct TmemLd;
+template <> struct TmemLd<16> {
+  static __device__ __forceinline__ void ld(uint32_t taddr, uint32_t* v) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                 : "r"(taddr) : "memory");
+  }
+};
+template <> struct TmemLd<32> {
+  static __device__ __forceinline__ void ld(uint32_t taddr, uint32_t* v) {
+    TmemLd<16>::ld(taddr, v);
+    TmemLd<16>::ld(taddr + 16, v + 16);
+  }
+};
+template <> struct TmemLd<64> {
+  static __device__ __forceinline__ void ld(uint32_t taddr, uint32_t* v) {
+    TmemLd<32>::ld(taddr, v);
+    TmemLd<32>::ld(taddr + 32, v + 32);
+  }
+};
+
+// CTA c of G owns tiles [c*T/G, (c+1)*T/G); the CTA that owns tile t:
+__device__ __forceinline__ long long range_begin(long long c, long long T, long long G) { return c * T / G; }
+__device__ __forceinline__ int owner_of(long long t, long long T, long long G) { return static_cast<int>(((t + 1) * G - 1) / T); }
+
+// ---------------------------------------------------------------------------------------------
+// The kernel
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
+  uint16_t v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts_u16(uint32_t addr, uint32_t v) {
+  asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(static_cast<uint16_t>(v)) : "memory");
+}
+__device__ __forceinline__ void sts_zero16B(uint32_t addr) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+}
+
+// Algorithm 1 for one chain, kBatch delta bytes at a time.  `pos` carries offset_t in its low and
+// offset_r in its high 16 bits, so one add advances both cursors.  Within a batch all positions
+// are formed first, then all W_t loads are issued, then all stores, so that the shared-memory
+// round trips of different entries overlap.
+constexpr int kBatch = 8;
+
+__device__ __forceinline__ void decode_chain(uint32_t stage, uint32_t wr, uint32_t hdr, uint32_t code_addr, uint32_t len) {
+  if (hdr == 0xFFFFFFFFu) return;                       // empty chain
+  uint32_t pos = hdr;
+  {                                                     // first pair: absolute 16-bit positions
+    const uint32_t at = stage + swizzled_offset(pos & 0xFFFFu);
+    const uint32_t v = lds_u16(at);
+    sts_u16(at, 0);                                     // W_t[offset_t] = 0
+    sts_u16(wr + swizzled_offset(pos >> 16), v);        // W_r[offset_r] = W_t[offset_t]
+  }
+  uint32_t word_addr = code_addr & ~3u;
+  const uint32_t shift = (code_addr & 3u) * 8u;
+  for (uint32_t k0 = 0; k0 < len; k0 += kBatch) {
+    const uint32_t w0 = lds_u32(word_addr), w1 = lds_u32(word_addr + 4), w2 = lds_u32(word_addr + 8);
+    word_addr += kBatch;
+    const uint32_t bytes[2] = {__funnelshift_r(w0, w1, shift), __funnelshift_r(w1, w2, shift)};
+    uint32_t at[kBatch], ar[kBatch], val[kBatch];
+    bool real[kBatch];
+#pragma unroll
+    for (int q = 0; q < kBatch; ++q) {
+      uint32_t bt = (bytes[q >> 2] >> (8 * (q & 3))) & 0xFFu;
+      bt = (k0 + q < len) ? bt : 0u;                    // past the end: behaves like a dummy
+      const uint32_t dt = bt & 0xFu, dr = bt >> 4;
+      pos += dt | (dr << 16);
+      real[q] = (dt != 0u) && (dr != 0u);               // a zero nibble marks a dummy point
+      at[q] = stage + swizzled_offset(pos & 0xFFFFu);
+      ar[q] = wr + swizzled_offset(pos >> 16);
+    }
+#pragma unroll
+    for (int q = 0; q < kBatch; ++q)
+      if (real[q]) val[q] = lds_u16(at[q]);
+#pragma unroll
+    for (int q = 0; q < kBatch; ++q)
+      if (real[q]) { sts_u16(at[q], 0); sts_u16(ar[q], val[q]); }
+  }
+}
+
+template <int NPAD>
+__global__ void __launch_bounds__(kThreads, 1)
+tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int S = a.num_stages;
+  uint8_t* wr_base = smem + static_cast<size_t>(S) * a.stage_stride;           // kGroups x 16 KB
+  uint8_t* bar_base = wr_base + kGroups * kWrBytes;
+  // barrier block: full[8] mma_done[8] decoded[8] acc_full[2] acc_empty[2] | tmem slot | flags
+  uint64_t* bars = reinterpret_cast<uint64_t*>(bar_base);
+  const uint32_t bar_full = smem_u32(bars), bar_mma = smem_u32(bars + 8), bar_dec = smem_u32(bars + 16);
+  const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 33);
+  volatile unsigned int* last_flag = reinterpret_cast<volatile unsigned int*>(bars + 34);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const long long T = a.total_tiles, G = gridDim.x;
+  const long long t_begin = range_begin(blockIdx.x, T, G), t_end = range_begin(blockIdx.x + 1, T, G);
+  const int n_tiles = static_cast<int>(t_end - t_begin);
+  const int kt_begin = static_cast<int>(t_begin % a.tiles_k);
+  const uint32_t smem_base = smem_u32(smem);
+
+  if (tid == 0) {
+    for (int s = 0; s < kMaxStages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_mma + 8 * s, 1);
+      mbar_init(bar_dec + 8 * s, 128);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_accfull + 8 * b, 1);
+      mbar_init(bar_accempty + 8 * b, 128);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kAllocWarp) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const WaitCtx wctx{abort_flag, a.status, global_timer()};
+
+  if (warp == kProducerWarp) {
+    // ------------------------------------------------------------------ producer
+    // The warp reads 32 directory entries at a time (one per lane); lane 0 issues the copies.
+    int issued = 0, s = 0, kt = kt_begin;
+    uint32_t ph = 0;                                            // phase of the stage's current use
+    bool alive = true;
+    for (int base = 0; base < n_tiles && alive; base += 32) {
+      uint4 mine = make_uint4(0, 0, 0, 0);
+      if (base + lane < n_tiles) mine = __ldg(reinterpret_cast<const uint4*>(a.dir + t_begin + base + lane));
+      const int cnt = n_tiles - base < 32 ? n_tiles - base : 32;
+      for (int j = 0; j < cnt; ++j) {
+        const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.x, j), bytes = __shfl_sync(0xFFFFFFFFu, mine.y, j);
+        if (lane == 0) {
+          const int i = base + j;
+          if (i >= S && !mbar_wait(bar_mma + 8 * s, ph ^ 1u, wctx, kStProducer)) alive = false;
+          if (alive) {
+            const uint32_t stage = smem_base + static_cast<uint32_t>(s) * a.stage_stride;
+            const uint32_t full = bar_full + 8 * s;
+            mbar_arrive_expect_tx(full, bytes + 128u * NPAD * 2u);
+            bulk_copy_g2s(stage, a.blob + static_cast<size_t>(off16) * 16, bytes, full);
+            tma_load_2d(stage + a.x_offset, &x_map, 0, kt * kTileK, full);
+            issued = i + 1;
+          }
+        }
+        alive = __shfl_sync(0xFFFFFFFFu, alive ? 1 : 0, 0) != 0;
+        if (!alive) break;
+        if (++s == S) { s = 0; ph ^= 1u; }
+        if (++kt == a.tiles_k) kt = 0;
+      }
+    }
+    if (lane == 0 && *abort_flag) {
+      // let the copies still in flight land before the CTA goes away
+      const int first = issued > S ? issued - S : 0;
+      for (int i = first; i < issued; ++i) {
+        const uint32_t full = bar_full + 8 * (i % S);
+        const unsigned long long t1 = global_timer();
+        while (!mbar_try_wait(full, (i / S) & 1)) {
+          if (global_timer() - t1 > kWaitLimitNs / 4) { atomicCAS(a.status, 0u, (uint32_t)kStDrain); break; }
+        }
+      }
+    }
+  } else if (warp == kMmaWarp) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      // instruction descriptor: sparse, D = f32, A = B = f16, A K-major, B MN-major, N = NPAD, M = 128
+      const uint32_t idesc = (1u << 2) | (1u << 4) | (1u << 16) | (static_cast<uint32_t>(NPAD >> 3) << 17) | (8u << 24);
+      // A: K-major, 128-byte swizzle, 8-row groups 1024 B apart
+      const uint64_t adesc_hi = (uint64_t(1) << 16) | (uint64_t(1024 >> 4) << 32) | (uint64_t(1) << 46) | (uint64_t(2) << 61);
+      // B: X block, k rows of NPAD*2 bytes, swizzle span = row pitch, 8-row groups 8*pitch apart
+      constexpr uint64_t kBLayout = NPAD == 16 ? 6 : NPAD == 32 ? 4 : 2;
+      const uint64_t bdesc_hi = (uint64_t(1) << 16) | (uint64_t((8 * NPAD * 2) >> 4) << 32) | (uint64_t(1) << 46) | (kBLayout << 61);
+      const uint32_t wr0 = smem_u32(wr_base);
+      int seg = 0, s = 0, kt = kt_begin;
+      uint32_t ph = 0;
+      for (int i = 0; i < n_tiles; ++i) {
+        const bool first_of_seg = (i == 0) || (kt == 0);
+        const bool last_of_seg = (i == n_tiles - 1) || (kt == a.tiles_k - 1);
+        const int b = seg & 1, g = i & 1;
+        if (first_of_seg && (seg >> 1) >= 1 &&
+            !mbar_wait(bar_accempty + 8 * b, ((seg >> 1) - 1) & 1, wctx, kStMmaAccEmpty)) break;
+        if (!mbar_wait(bar_dec + 8 * s, ph, wctx, kStMmaDecoded)) break;
+        tc_fence_after();
+        const uint32_t stage = smem_base + static_cast<uint32_t>(s) * a.stage_stride;
+        const uint32_t wr = wr0 + g * kWrBytes;
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(b * NPAD);
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+          const uint64_t bdesc = bdesc_hi | (((stage + a.x_offset + kb * 32 * NPAD * 2) & 0x3FFFFu) >> 4);
+          const uint32_t id = idesc | static_cast<uint32_t>(kb & 1);
+          umma_sp_f16(d_tmem, adesc_hi | (((stage + kb * 32) & 0x3FFFFu) >> 4), bdesc,
+                      tmem_base + kColMetaT + 4 * g + (kb & ~1), id, (first_of_seg && kb == 0) ? 0u : 1u);
+          umma_sp_f16(d_tmem, adesc_hi | (((wr + kb * 32) & 0x3FFFFu) >> 4), bdesc,
+                      tmem_base + kColMetaR, id, 1u);
+        }
+        umma_commit(bar_mma + 8 * s);       // frees the stage, this group's W_r and metadata columns
+        if (last_of_seg) { umma_commit(bar_accfull + 8 * b); ++seg; }
+        if (++s == S) { s = 0; ph ^= 1u; }
+        if (++kt == a.tiles_k) kt = 0;
+      }
+    }
+  } else if (warp >= kDecodeWarp0 && warp < kEpilogueWarp0) {
+    // ------------------------------------------------------------------ decode (Algorithm 1)
+    const int g = (warp - kDecodeWarp0) >> 2;
+    const int r = tid - (kDecodeWarp0 + 4 * g) * 32;            // chain / row / tensor-memory lane 0..127
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const uint32_t wr = smem_u32(wr_base + g * kWrBytes);
+    if (g == 0) {   // constant metadata of W_r: every window selects in-window positions {2, 3}
+      asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};"
+                   ::"r"(tmem_base + lane_base + kColMetaR), "r"(0xEEEEEEEEu), "r"(0xEEEEEEEEu) : "memory");
+    }
+    int s = g % S, prev_s = 0;
+    uint32_t ph = (g / S) & 1, prev_ph = 0;
+    for (int i = g; i < n_tiles; i += kGroups) {
+      // W_r and the metadata columns of this group were last read by the MMAs of tile i - 2
+      bool ok = (i < kGroups) || mbar_wait(bar_mma + 8 * prev_s, prev_ph, wctx, kStDecodeWrFree);
+      if (ok) {   // clear W_r: thread r clears row r (its own chain writes only there)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) sts_zero16B(wr + r * 128 + c * 16);
+      }
+      ok = ok && mbar_wait(bar_full + 8 * s, ph, wctx, kStDecodeFull);
+      // Residual entries land in any row, so the whole of W_r must be clear before anyone
+      // scatters; the same barrier makes the give-up decision uniform across the group.
+      if (!named_bar_all(1 + g, 128, ok)) break;
+      const uint32_t stage = smem_base + static_cast<uint32_t>(s) * a.stage_stride;
+      // metadata -> tensor memory (4 columns of this group)
+      {
+        uint32_t m0, m1, m2, m3;
+        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(m0), "=r"(m1), "=r"(m2), "=r"(m3) : "r"(stage + kMetaOff + r * 16));
+        asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
+                     ::"r"(tmem_base + lane_base + kColMetaT + 4 * g), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
+      }
+      // byte offset of this thread's chain = exclusive prefix sum of the chain lengths.
+      // Each warp scans all 128 lengths (4 per lane) with shuffles; no cross-warp exchange.
+      uint32_t off, len;
+      {
+        const uint32_t quad = lds_u32(stage + kLenOff + lane * 4);
+        const uint32_t qsum = __dp4a(quad, 0x01010101u, 0u);
+        uint32_t incl = qsum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+          if (lane >= d) incl += n;
+        }
+        const int src = r >> 2;                                  // lane that holds my quad
+        const uint32_t q = __shfl_sync(0xFFFFFFFFu, quad, src);
+        const uint32_t excl = __shfl_sync(0xFFFFFFFFu, incl - qsum, src);
+        const int sub = r & 3;
+        off = excl + __dp4a(q & ((1u << (8 * sub)) - 1u), 0x01010101u, 0u);
+        len = (q >> (8 * sub)) & 0xFFu;
+      }
+      decode_chain(stage, wr, lds_u32(stage + kHdrOff + r * 4), stage + kPddOff + off, len);
+      // Residual layer: (position, value) entries go to W_r too
+      {
+        const uint32_t pdd_len = lds_u32(stage + kInfoOff), res_cnt = lds_u32(stage + kInfoOff + 4);
+        const uint32_t res = stage + kPddOff + ((pdd_len + 3u) & ~3u);
+        for (uint32_t k = r; k < res_cnt; k += 128) {
+          const uint32_t rv = lds_u32(res + 4 * k);
+          sts_u16(wr + swizzled_offset(rv & 0xFFFFu), rv >> 16);
+        }
+      }
+      fence_proxy_async_smem();                                   // generic-proxy writes -> MMA reads
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      tc_fence_before();
+      mbar_arrive(bar_dec + 8 * s);
+      prev_s = s; prev_ph = ph;
+      s += kGroups;
+      if (s >= S) { s -= S; ph ^= 1u; }
+    }
+  } else if (warp >= kEpilogueWarp0) {
+    // ------------------------------------------------------------------ epilogue
+    const int et = tid - kEpilogueWarp0 * 32;                    // 0..127 = row of the tile = tensor-memory lane
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    int seg = 0;
+    long long t = t_begin;
+    while (t < t_end) {
+      const int mt = static_cast<int>(t / a.tiles_k);
+      const long long row_tile_begin = static_cast<long long>(mt) * a.tiles_k, row_tile_end = row_tile_begin + a.tiles_k;
+      const long long seg_end = row_tile_end < t_end ? row_tile_end : t_end;
+      const bool complete = (t == row_tile_begin) && (seg_end == row_tile_end);
+      const int b = seg & 1;
+      if (!named_bar_all(3, 128, mbar_wait(bar_accfull + 8 * b, (seg >> 1) & 1, wctx, kStEpilogueAccFull))) break;
+      tc_fence_after();
+      uint32_t v[NPAD];
+      TmemLd<NPAD>::ld(tmem_base + lane_base + static_cast<uint32_t>(b * NPAD), v);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      tc_fence_before();
+      mbar_arrive(bar_accempty + 8 * b);
+      const int row = mt * kTileM + et;
+      bool write_y = complete;
+      if (!complete) {
+        // partial sums: slot 2*cta + (this row-tile is not the first one of my range)
+        const int slot = 2 * blockIdx.x + (t_begin < row_tile_begin ? 1 : 0);
+        float* mine = a.partials + static_cast<size_t>(slot) * NPAD * 128 + et;
+#pragma unroll
+        for (int c = 0; c < NPAD; ++c) __stcg(mine + c * 128, __uint_as_float(v[c]));
+        __threadfence();
+        named_bar_sync(3, 128);
+        const int c_first = owner_of(row_tile_begin, T, G), c_last = owner_of(row_tile_end - 1, T, G);
+        if (et == 0) {
+          const unsigned int old = atomicAdd(a.counters + mt, 1u);
+          const bool last = old == static_cast<unsigned int>(c_last - c_first);
+          if (last) a.counters[mt] = 0;                          // leave the workspace cleared
+          *last_flag = last ? 1u : 0u;
+        }
+        named_bar_sync(3, 128);
+        if (*last_flag) {
+          __threadfence();
+          float acc[NPAD];
+#pragma unroll
+          for (int c = 0; c < NPAD; ++c) acc[c] = 0.f;
+          for (int c_id = c_first; c_id <= c_last; ++c_id) {      // fixed order: deterministic sum
+            const int sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
+            const float* p = a.partials + static_cast<size_t>(sl) * NPAD * 128 + et;
+#pragma unroll
+            for (int c = 0; c < NPAD; ++c) acc[c] += __ldcg(p + c * 128);
+          }
+#pragma unroll
+          for (int c = 0; c < NPAD; ++c) v[c] = __float_as_uint(acc[c]);
+          write_y = true;
+        }
+        named_bar_sync(3, 128);                                   // last_flag may be rewritten next segment
+      }
+      if (write_y && row < a.M) {
+        __half* y = a.Y + static_cast<long long>(row) * a.ldy;
+        if (a.N == NPAD && (a.ldy & 7) == 0 && (reinterpret_cast<uintptr_t>(a.Y) & 15) == 0) {
+#pragma unroll
+          for (int c = 0; c < NPAD; c += 8) {
+            uint4 o;
+            __half2 h0 = __floats2half2_rn(__uint_as_float(v[c + 0]), __uint_as_float(v[c + 1]));
+            __half2 h1 = __floats2half2_rn(__uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
+            __half2 h2 = __floats2half2_rn(__uint_as_float(v[c + 4]), __uint_as_float(v[c + 5]));
+            __half2 h3 = __floats2half2_rn(__uint_as_float(v[c + 6]), __uint_as_float(v[c + 7]));
+            o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
+            o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
+            *reinterpret_cast<uint4*>(y + c) = o;
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < NPAD; ++c)
+            if (c < a.N) y[c] = __float2half_rn(__uint_as_float(v[c]));
+        }
+      }
+      ++seg;
+      t = seg_end;
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == kAllocWarp) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+struct DeviceInfo {
+  int sm_count = 0;
+  int cc_major = 0;
+  bool ok = false;
+};
+
+static int device_info(DeviceInfo* out) {
+  int dev = 0;
+  TL3_CUDA(cudaGetDevice(&dev));
+  static std::mutex mu;
+  static std::vector<DeviceInfo> cache;
+  std::lock_guard<std::mutex> lock(mu);
+  if (static_cast<size_t>(dev) >= cache.size()) cache.resize(dev + 1);
+  DeviceInfo& d = cache[dev];
+  if (!d.ok) {
+    TL3_CUDA(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev));
+    TL3_CUDA(cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+    d.ok = true;
+  }
+  *out = d;
+  return TL3_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+static inline int n_pad_of(int N) { return N <= 16 ? 16 : N <= 32 ? 32 : 64; }
+
+struct WorkspaceLayout {
+  size_t status_off = 0, counters_off = 256, partials_off = 0, total = 0;
+};
+
+static WorkspaceLayout workspace_layout(const tl3_matrix* m, int n_pad, int sm_count) {
+  WorkspaceLayout w;
+  w.partials_off = (256 + static_cast<size_t>(m->tiles_m) * 4 + 4095) / 4096 * 4096;
+  w.total = w.partials_off + static_cast<size_t>(2) * sm_count * n_pad * 128 * sizeof(float);
+  return w;
+}
+
+template <int NPAD>
+static int launch(const CUtensorMap& map, const KernelArgs& args, int grid, uint32_t smem_bytes, cudaStream_t stream) {
+  static bool configured = false;   // per template instance; same value every time
+  if (!configured) {
+    TL3_CUDA(cudaFuncSetAttribute(tl3_spmm_kernel<NPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemLimit)));
+    configured = true;
+  }
+  tl3_spmm_kernel<NPAD><<<grid, kThreads, smem_bytes, stream>>>(map, args);
+  TL3_CUDA(cudaGetLastError());
+  return TL3_OK;
+}
+
+}  // namespace tl3
+
+extern "C" {
+
+size_t tl3_device_bytes(const tl3_matrix* m) {
+  if (!m) return 0;
+  return tl3::plan_device_layout(const_cast<tl3_matrix*>(m));
+}
+
+int tl3_upload(tl3_matrix* m, void* dptr, void* stream) {
+  if (!m || !dptr || (reinterpret_cast<uintptr_t>(dptr) & 255) != 0) return TL3_ERR_INVALID_ARG;
+  if (m->p.tile_m != tl3::kTileM || m->p.tile_k != tl3::kTileK) return TL3_ERR_UNSUPPORTED;
+  const size_t bytes = tl3::plan_device_layout(m);
+  std::vector<uint8_t> staging;
+  try {
+    staging.resize(bytes);
+  } catch (const std::bad_alloc&) {
+    return TL3_ERR_NO_MEMORY;
+  }
+  tl3::pack_device_blob(m, staging.data());
+  // pageable source: the runtime returns once the data sits in its own staging buffers
+  TL3_CUDA(cudaMemcpyAsync(dptr, staging.data(), bytes, cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)));
+  m->dptr = dptr;
+  return TL3_OK;
+}
+
+size_t tl3_workspace_bytes(const tl3_matrix* m, int N) {
+  if (!m || N < 1 || N > 64) return 0;
+  tl3::DeviceInfo di;
+  if (tl3::device_info(&di) != TL3_OK) return 0;
+  return tl3::workspace_layout(m, tl3::n_pad_of(N), di.sm_count).total;
+}
+
+int tl3_workspace_init(void* workspace, size_t bytes, void* stream) {
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return TL3_ERR_INVALID_ARG;
+  TL3_CUDA(cudaMemsetAsync(workspace, 0, bytes, static_cast<cudaStream_t>(stream)));
+  return TL3_OK;
+}
+
+int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N, void* workspace, void* stream) {
+  using namespace tl3;
+  if (!m || !X || !Y || !workspace) return TL3_ERR_INVALID_ARG;
+  if (!m->dptr) return TL3_ERR_NOT_UPLOADED;
+  if (N < 1 || N > 64) return TL3_ERR_UNSUPPORTED;
+  if (ldx < N || ldy < N || (ldx & 7) != 0 || (reinterpret_cast<uintptr_t>(X) & 15) != 0 ||
+      (reinterpret_cast<uintptr_t>(Y) & 1) != 0 || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0)
+    return TL3_ERR_INVALID_ARG;
+  DeviceInfo di;
+  if (int rc = device_info(&di)) return rc;
+  if (di.cc_major != 10) return TL3_ERR_UNSUPPORTED;
+  const int n_pad = n_pad_of(N);
+
+  // shared-memory plan
+  // + 16: the decoder fetches delta bytes in aligned words and may read a few bytes past a block
+  const uint32_t block_area = (m->max_block_bytes + 16u + 1023u) / 1024u * 1024u;
+  const uint32_t x_bytes = 128u * n_pad * 2u;
+  const uint32_t stage_stride = block_area + x_bytes;
+  const uint32_t fixed = kGroups * kWrBytes + kBarrierBytes + 1024u;   // + alignment slack
+  if (fixed + 2u * stage_stride > kSmemLimit) return TL3_ERR_UNSUPPORTED;
+  int stages = static_cast<int>((kSmemLimit - fixed) / stage_stride);
+  if (stages > kMaxStages) stages = kMaxStages;
+  const uint32_t smem_bytes = fixed + static_cast<uint32_t>(stages) * stage_stride;
+
+  // tensor map of X: dims {N, K}, box {n_pad, 128}; columns >= N and rows >= K read as zero
+  EncodeTiledFn encode = encode_tiled_fn();
+  if (!encode) return TL3_ERR_UNSUPPORTED;
+  CUtensorMap map;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(m->K)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ldx) * 2};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(n_pad), 128};
+  const cuuint32_t elem_strides[2] = {1, 1};
+  const CUtensorMapSwizzle swz = n_pad == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : n_pad == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
+  const CUresult cr = encode(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(X), dims, strides, box, elem_strides,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (cr != CUDA_SUCCESS) { set_cuda_error(static_cast<int>(cr)); return TL3_ERR_CUDA; }
+
+  const long long total = m->n_tiles;
+  const int grid = static_cast<int>(total < di.sm_count ? total : di.sm_count);
+  const WorkspaceLayout wl = workspace_layout(m, n_pad, di.sm_count);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  KernelArgs args;
+  args.blob = static_cast<const uint8_t*>(m->dptr);
+  args.dir = reinterpret_cast<const DirEntry*>(args.blob + m->dir_offset);
+  args.total_tiles = total;
+  args.tiles_m = static_cast<int>(m->tiles_m);
+  args.tiles_k = static_cast<int>(m->tiles_k);
+  args.M = static_cast<int>(m->M);
+  args.N = N;
+  args.ldy = ldy;
+  args.Y = static_cast<__half*>(Y);
+  args.partials = reinterpret_cast<float*>(ws + wl.partials_off);
+  args.counters = reinterpret_cast<unsigned int*>(ws + wl.counters_off);
+  args.status = reinterpret_cast<unsigned int*>(ws + wl.status_off);
+  args.stage_stride = stage_stride;
+  args.x_offset = block_area;
+  args.num_stages = stages;
+  m->last_ctas = grid; m->last_stages = stages; m->last_smem = static_cast<int>(smem_bytes);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  switch (n_pad) {
+    case 16: return launch<16>(map, args, grid, smem_bytes, st);
+    case 32: return launch<32>(map, args, grid, smem_bytes, st);
+    default: return launch<64>(map, args, grid, smem_bytes, st);
+  }
+}
+
+int tl3_spmm_host(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int N, void* dX, void* dY, void* workspace, void* stream) {
+  if (!m || !X || !Y || !dX || !dY) return TL3_ERR_INVALID_ARG;
+  if (N < 1 || N > 64) return TL3_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // device copy of X with a leading dimension that satisfies the 16-byte rule
+  const int64_t ldx = (N + 7) / 8 * 8;
+  TL3_CUDA(cudaMemcpy2DAsync(dX, static_cast<size_t>(ldx) * 2, X, static_cast<size_t>(N) * 2, static_cast<size_t>(N) * 2,
+                             static_cast<size_t>(m->K), cudaMemcpyHostToDevice, st));
+  if (int rc = tl3_spmm(m, dX, ldx, dY, N, N, workspace, stream)) return rc;
+  TL3_CUDA(cudaMemcpyAsync(Y, dY, static_cast<size_t>(m->M) * N * 2, cudaMemcpyDeviceToHost, st));
+  TL3_CUDA(cudaStreamSynchronize(st));
+  return TL3_OK;
+}
+
+int tl3_status(const tl3_matrix* m, void* workspace, void* stream) {
+  (void)m;
+  if (!workspace) return TL3_ERR_INVALID_ARG;
+  unsigned int st = 0;
+  TL3_CUDA(cudaMemcpyAsync(&st, workspace, sizeof(st), cudaMemcpyDeviceToHost, static_cast<cudaStream_t>(stream)));
+  TL3_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+  return st == 0 ? TL3_OK : TL3_ERR_DEVICE_TIMEOUT;
+}
+
+int tl3_last_launch(const tl3_matrix* m, int* ctas, int* stages, int* smem_bytes) {
+  if (!m) return TL3_ERR_INVALID_ARG;
+  if (ctas) *ctas = m->last_ctas;
+  if (stages) *stages = m->last_stages;
+  if (smem_bytes) *smem_bytes = m->last_smem;
+  return TL3_OK;
+}
+
+int tl3_last_cuda_error(void) { return tl3::g_last_cuda_error; }
+
+}  // extern "C"
