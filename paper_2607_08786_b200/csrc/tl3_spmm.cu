@@ -25,6 +25,7 @@
 #include <cuda_fp16.h>
 
 #include <cstdint>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <vector>
@@ -48,18 +49,21 @@ void set_cuda_error(int e) { g_last_cuda_error = e; }
 // ---------------------------------------------------------------------------------------------
 // Kernel configuration
 // ---------------------------------------------------------------------------------------------
-constexpr int kThreads = 512;             // 16 warps
+constexpr int kGroups = 4;                // decode groups of four warps; tile i goes to group i % 4
 constexpr int kProducerWarp = 0;
 constexpr int kMmaWarp = 1;
-constexpr int kAllocWarp = 2;
-constexpr int kDecodeWarp0 = 4;           // warps 4-7: decode group 0, warps 8-11: group 1
-constexpr int kEpilogueWarp0 = 12;        // warps 12-15
-constexpr int kGroups = 2;
+constexpr int kAllocWarp = 2;             // warp 3 is idle; decode groups start at a multiple of four warps
+                                          // because a warp reaches tensor-memory lanes 32*(warp%4)..+31
+constexpr int kDecodeWarp0 = 4;           // warps 4-7: decode group 0, 8-11: group 1, ...
+constexpr int kEpilogueWarp0 = kDecodeWarp0 + 4 * kGroups;
+constexpr int kThreads = (kEpilogueWarp0 + 4) * 32;
 constexpr int kMaxStages = 8;
 constexpr uint32_t kWrBytes = 16384;
+constexpr int kWrBuffers = 4;             // W_r ring: tile i uses buffer i % 4
+static_assert(kWrBuffers % kGroups == 0, "a W_r buffer must always belong to the same decode group");
 constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColMetaT = 128;       // + 4 * group
-constexpr uint32_t kColMetaR = 136;       // two columns of 0xEEEEEEEE
+constexpr uint32_t kColMetaT = 128;       // + 4 * (tile % 4): metadata of W_t, four columns per tile in flight
+constexpr uint32_t kColMetaR = 144;       // two columns of 0xEEEEEEEE
 constexpr uint32_t kSmemLimit = 232448;   // 227 KB
 constexpr uint32_t kBarrierBytes = 1024;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per kernel
@@ -84,7 +88,26 @@ struct KernelArgs {
   uint32_t stage_stride;     // bytes per stage (block area + X tile), multiple of 1024
   uint32_t x_offset;         // offset of the X tile inside a stage, multiple of 1024
   int num_stages;
+  long long* timing;         // phase-timing buffer (debug builds), else null
+  int debug_skip;            // debug builds: bit 0 skips the W_t MMAs, bit 1 the W_r MMAs, bit 2 the chain decode
 };
+
+// Optional per-role phase timing (build with -DTL3_PHASE_TIMING): CTA 0 adds the clock cycles it
+// spends between TL3_TACC marks into a buffer set with tl3_debug_set_timing_buffer().
+#ifdef TL3_PHASE_TIMING
+static long long* g_timing_buffer = nullptr;
+#define TL3_T0() long long tacc_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long tprev_ = clock64();
+#define TL3_TACC(k) { const long long tn_ = clock64(); tacc_[k] += tn_ - tprev_; tprev_ = tn_; }
+#define TL3_TDUMP(base) { if (a.timing && blockIdx.x == 0) for (int q_ = 0; q_ < 8; ++q_) a.timing[(base) + q_] = tacc_[q_]; }
+#define TL3_SKIP(bit) (a.debug_skip & (bit))
+#define TL3_STAMP(tile, k) { if (a.timing && blockIdx.x == 0 && (tile) >= 18 && (tile) < 26) a.timing[200 + 8 * ((tile) - 18) + (k)] = clock64(); }
+#else
+#define TL3_SKIP(bit) false
+#define TL3_STAMP(tile, k) {}
+#define TL3_T0() {}
+#define TL3_TACC(k) {}
+#define TL3_TDUMP(base) {}
+#endif
 
 // ---------------------------------------------------------------------------------------------
 // PTX helpers
@@ -106,13 +129,16 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// One probe of the barrier phase.  The hint lets the hardware park the thread (up to that many
+// nanoseconds, or until the phase completes) instead of spinning, so waiting warps do not take
+// issue slots from the warps that have work.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t done;
   asm volatile(
       "{\n\t.reg .pred q;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, q;\n\t}"
-      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+      : "=r"(done) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
   return done != 0;
 }
 
@@ -128,7 +154,7 @@ struct WaitCtx {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w, uint32_t code) {
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 255u) {
+    if ((it & 15u) == 15u) {
       if (*w.abort_flag) return false;
       if (global_timer() - w.t0 > kWaitLimitNs) {
         atomicCAS(w.status, 0u, code);
@@ -168,12 +194,25 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
                ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
 
-__device__ __forceinline__ void umma_sp_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t e_tmem,
-                                            uint32_t idesc, uint32_t accumulate) {
+// One lane of a converged warp; the caller keeps every operand warp-uniform so that the
+// single-thread instructions (bulk copies, MMAs, commits) take uniform registers directly.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+
+// D[tmem] (+)= A_sparse[smem] * B[smem] with the 2-bit metadata at e_tmem.  The shared-memory
+// descriptors are passed as their low words (start address field) and one common high word each.
+__device__ __forceinline__ void umma_sp_f16(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                            uint32_t e_tmem, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-      "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %7, 0;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], da, db, [%5], %6, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -277,8 +316,8 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int S = a.num_stages;
-  uint8_t* wr_base = smem + static_cast<size_t>(S) * a.stage_stride;           // kGroups x 16 KB
-  uint8_t* bar_base = wr_base + kGroups * kWrBytes;
+  uint8_t* wr_base = smem + static_cast<size_t>(S) * a.stage_stride;           // kWrBuffers x 16 KB
+  uint8_t* bar_base = wr_base + kWrBuffers * kWrBytes;
   // barrier block: full[8] mma_done[8] decoded[8] acc_full[2] acc_empty[2] | tmem slot | flags
   uint64_t* bars = reinterpret_cast<uint64_t*>(bar_base);
   const uint32_t bar_full = smem_u32(bars), bar_mma = smem_u32(bars + 8), bar_dec = smem_u32(bars + 16);
@@ -319,34 +358,41 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
 
   if (warp == kProducerWarp) {
     // ------------------------------------------------------------------ producer
-    // The warp reads 32 directory entries at a time (one per lane); lane 0 issues the copies.
+    // The whole warp runs the loop with warp-uniform state; one elected lane issues the copies.
+    // Directory entries are read 32 at a time (one per lane) and broadcast with shuffles.
     int issued = 0, s = 0, kt = kt_begin;
     uint32_t ph = 0;                                            // phase of the stage's current use
+    uint32_t stage = smem_base;
     bool alive = true;
+    TL3_T0()
     for (int base = 0; base < n_tiles && alive; base += 32) {
       uint4 mine = make_uint4(0, 0, 0, 0);
       if (base + lane < n_tiles) mine = __ldg(reinterpret_cast<const uint4*>(a.dir + t_begin + base + lane));
       const int cnt = n_tiles - base < 32 ? n_tiles - base : 32;
       for (int j = 0; j < cnt; ++j) {
         const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.x, j), bytes = __shfl_sync(0xFFFFFFFFu, mine.y, j);
-        if (lane == 0) {
-          const int i = base + j;
-          if (i >= S && !mbar_wait(bar_mma + 8 * s, ph ^ 1u, wctx, kStProducer)) alive = false;
-          if (alive) {
-            const uint32_t stage = smem_base + static_cast<uint32_t>(s) * a.stage_stride;
-            const uint32_t full = bar_full + 8 * s;
-            mbar_arrive_expect_tx(full, bytes + 128u * NPAD * 2u);
-            bulk_copy_g2s(stage, a.blob + static_cast<size_t>(off16) * 16, bytes, full);
-            tma_load_2d(stage + a.x_offset, &x_map, 0, kt * kTileK, full);
-            issued = i + 1;
-          }
-        }
-        alive = __shfl_sync(0xFFFFFFFFu, alive ? 1 : 0, 0) != 0;
+        const int i = base + j;
+        TL3_TACC(0)
+        if (i >= S) alive = __all_sync(0xFFFFFFFFu, mbar_wait(bar_mma + 8 * s, ph ^ 1u, wctx, kStProducer));
+        TL3_TACC(1)
         if (!alive) break;
-        if (++s == S) { s = 0; ph ^= 1u; }
+        if (lane == 0) TL3_STAMP(i, 0)
+        const uint32_t full = bar_full + 8 * s;
+        const uint8_t* src = a.blob + static_cast<size_t>(off16) * 16;
+        if (elect_one()) {
+          mbar_arrive_expect_tx(full, bytes + (TL3_SKIP(64) ? 0u : 128u * NPAD * 2u));
+          bulk_copy_g2s(stage, src, bytes, full);
+          if (!TL3_SKIP(64)) tma_load_2d(stage + a.x_offset, &x_map, 0, kt * kTileK, full);
+          TL3_STAMP(i, 1)
+        }
+        __syncwarp();
+        issued = i + 1;
+        stage += a.stage_stride;
+        if (++s == S) { s = 0; ph ^= 1u; stage = smem_base; }
         if (++kt == a.tiles_k) kt = 0;
       }
     }
+    if (lane == 0) TL3_TDUMP(0)
     if (lane == 0 && *abort_flag) {
       // let the copies still in flight land before the CTA goes away
       const int first = issued > S ? issued - S : 0;
@@ -360,73 +406,101 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     }
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      // instruction descriptor: sparse, D = f32, A = B = f16, A K-major, B MN-major, N = NPAD, M = 128
-      const uint32_t idesc = (1u << 2) | (1u << 4) | (1u << 16) | (static_cast<uint32_t>(NPAD >> 3) << 17) | (8u << 24);
-      // A: K-major, 128-byte swizzle, 8-row groups 1024 B apart
-      const uint64_t adesc_hi = (uint64_t(1) << 16) | (uint64_t(1024 >> 4) << 32) | (uint64_t(1) << 46) | (uint64_t(2) << 61);
-      // B: X block, k rows of NPAD*2 bytes, swizzle span = row pitch, 8-row groups 8*pitch apart
-      constexpr uint64_t kBLayout = NPAD == 16 ? 6 : NPAD == 32 ? 4 : 2;
-      const uint64_t bdesc_hi = (uint64_t(1) << 16) | (uint64_t((8 * NPAD * 2) >> 4) << 32) | (uint64_t(1) << 46) | (kBLayout << 61);
-      const uint32_t wr0 = smem_u32(wr_base);
-      int seg = 0, s = 0, kt = kt_begin;
-      uint32_t ph = 0;
-      for (int i = 0; i < n_tiles; ++i) {
-        const bool first_of_seg = (i == 0) || (kt == 0);
-        const bool last_of_seg = (i == n_tiles - 1) || (kt == a.tiles_k - 1);
-        const int b = seg & 1, g = i & 1;
-        if (first_of_seg && (seg >> 1) >= 1 &&
-            !mbar_wait(bar_accempty + 8 * b, ((seg >> 1) - 1) & 1, wctx, kStMmaAccEmpty)) break;
-        if (!mbar_wait(bar_dec + 8 * s, ph, wctx, kStMmaDecoded)) break;
-        tc_fence_after();
-        const uint32_t stage = smem_base + static_cast<uint32_t>(s) * a.stage_stride;
-        const uint32_t wr = wr0 + g * kWrBytes;
-        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(b * NPAD);
+    // Warp-uniform loop; one elected lane issues the eight MMAs of a tile and the commits.
+    // instruction descriptor: sparse, D = f32, A = B = f16, A K-major, B MN-major, N = NPAD, M = 128
+    const uint32_t idesc = (1u << 2) | (1u << 4) | (1u << 16) | (static_cast<uint32_t>(NPAD >> 3) << 17) | (8u << 24);
+    // Shared-memory descriptors: low word = start address >> 4 (+ an unused leading-offset field),
+    // high word = stride between 8-row groups, descriptor version, swizzle mode.
+    // A: K-major, 128-byte swizzle, 8-row groups 1024 B apart; a 32-wide k-block is 32 bytes of a row.
+    // B: X block, k rows of NPAD*2 bytes, swizzle span = row pitch, 8-row groups 8*pitch apart;
+    //    a k-block is 32 rows.
+    constexpr uint32_t kAHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    constexpr uint32_t kBLayout = NPAD == 16 ? 6u : NPAD == 32 ? 4u : 2u;
+    constexpr uint32_t kBHi = ((8u * NPAD * 2u) >> 4) | (1u << 14) | (kBLayout << 29);
+    constexpr uint32_t kLboOne = 1u << 16;
+    constexpr uint32_t kAStep = 32u >> 4, kBStep = (32u * NPAD * 2u) >> 4;
+    const uint32_t a_lo0 = (smem_base >> 4) | kLboOne, stride16 = a.stage_stride >> 4, x16 = a.x_offset >> 4;
+    const uint32_t w_lo0 = (smem_u32(wr_base) >> 4) | kLboOne;
+    int seg = 0, s = 0, kt = kt_begin;
+    uint32_t ph = 0, a_lo = a_lo0;
+    TL3_T0()
+    for (int i = 0; i < n_tiles; ++i) {
+      const bool first_of_seg = (i == 0) || (kt == 0);
+      const bool last_of_seg = (i == n_tiles - 1) || (kt == a.tiles_k - 1);
+      const int b = seg & 1, wb = i & (kWrBuffers - 1);
+      bool ok = true;
+      if (first_of_seg && (seg >> 1) >= 1) ok = mbar_wait(bar_accempty + 8 * b, ((seg >> 1) - 1) & 1, wctx, kStMmaAccEmpty);
+      TL3_TACC(0)
+      ok = ok && mbar_wait(bar_dec + 8 * s, ph, wctx, kStMmaDecoded);
+      TL3_TACC(1)
+      if (!__all_sync(0xFFFFFFFFu, ok)) break;
+      if (lane == 0) TL3_STAMP(i, 4)
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(b * NPAD);
+      const uint32_t e_t = tmem_base + kColMetaT + 4 * wb, e_r = tmem_base + kColMetaR;
+      const uint32_t b_lo = a_lo + x16, w_lo = w_lo0 + wb * (kWrBytes >> 4);
+      const uint32_t mma_bar = bar_mma + 8 * s, acc_bar = bar_accfull + 8 * b;
+      if (elect_one()) {
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb) {
-          const uint64_t bdesc = bdesc_hi | (((stage + a.x_offset + kb * 32 * NPAD * 2) & 0x3FFFFu) >> 4);
           const uint32_t id = idesc | static_cast<uint32_t>(kb & 1);
-          umma_sp_f16(d_tmem, adesc_hi | (((stage + kb * 32) & 0x3FFFFu) >> 4), bdesc,
-                      tmem_base + kColMetaT + 4 * g + (kb & ~1), id, (first_of_seg && kb == 0) ? 0u : 1u);
-          umma_sp_f16(d_tmem, adesc_hi | (((wr + kb * 32) & 0x3FFFFu) >> 4), bdesc,
-                      tmem_base + kColMetaR, id, 1u);
+          if (!TL3_SKIP(1)) umma_sp_f16(d_tmem, a_lo + kb * kAStep, kAHi, b_lo + kb * kBStep, kBHi, e_t + (kb & ~1), id,
+                                        (first_of_seg && kb == 0) ? 0u : 1u);
+          if (!TL3_SKIP(2)) umma_sp_f16(d_tmem, w_lo + kb * kAStep, kAHi, b_lo + kb * kBStep, kBHi, e_r, id, 1u);
         }
-        umma_commit(bar_mma + 8 * s);       // frees the stage, this group's W_r and metadata columns
-        if (last_of_seg) { umma_commit(bar_accfull + 8 * b); ++seg; }
-        if (++s == S) { s = 0; ph ^= 1u; }
-        if (++kt == a.tiles_k) kt = 0;
+        umma_commit(mma_bar);         // frees the stage, this tile's W_r buffer and metadata columns
+        if (last_of_seg) umma_commit(acc_bar);
       }
+      __syncwarp();
+      if (lane == 0) TL3_STAMP(i, 5)
+      TL3_TACC(2)
+      if (last_of_seg) ++seg;
+      a_lo += stride16;
+      if (++s == S) { s = 0; ph ^= 1u; a_lo = a_lo0; }
+      if (++kt == a.tiles_k) kt = 0;
     }
+    if (lane == 0) TL3_TDUMP(8)
   } else if (warp >= kDecodeWarp0 && warp < kEpilogueWarp0) {
     // ------------------------------------------------------------------ decode (Algorithm 1)
     const int g = (warp - kDecodeWarp0) >> 2;
     const int r = tid - (kDecodeWarp0 + 4 * g) * 32;            // chain / row / tensor-memory lane 0..127
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const uint32_t wr = smem_u32(wr_base + g * kWrBytes);
+    const uint32_t wr0 = smem_u32(wr_base);
     if (g == 0) {   // constant metadata of W_r: every window selects in-window positions {2, 3}
       asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};"
                    ::"r"(tmem_base + lane_base + kColMetaR), "r"(0xEEEEEEEEu), "r"(0xEEEEEEEEu) : "memory");
     }
-    int s = g % S, prev_s = 0;
-    uint32_t ph = (g / S) & 1, prev_ph = 0;
-    for (int i = g; i < n_tiles; i += kGroups) {
-      // W_r and the metadata columns of this group were last read by the MMAs of tile i - 2
-      bool ok = (i < kGroups) || mbar_wait(bar_mma + 8 * prev_s, prev_ph, wctx, kStDecodeWrFree);
-      if (ok) {   // clear W_r: thread r clears row r (its own chain writes only there)
+    constexpr int kHist = kWrBuffers / kGroups;                  // own tiles between two uses of a W_r buffer
+    int s = g % S, hist_s[kHist];
+    uint32_t ph = (g / S) & 1, hist_ph[kHist];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) sts_zero16B(wr + r * 128 + c * 16);
+    for (int h = 0; h < kHist; ++h) { hist_s[h] = 0; hist_ph[h] = 0; }
+    TL3_T0()
+    for (int i = g; i < n_tiles; i += kGroups) {
+      TL3_TACC(0)
+      const int wb = i & (kWrBuffers - 1);
+      const uint32_t wr = wr0 + wb * kWrBytes;
+      // this W_r buffer and its metadata columns were last read by the MMAs of tile i - 4
+      bool ok = (i < kWrBuffers) || mbar_wait(bar_mma + 8 * hist_s[kHist - 1], hist_ph[kHist - 1], wctx, kStDecodeWrFree);
+      TL3_TACC(1)
+      if (ok && !TL3_SKIP(8)) {   // clear W_r, 16 bytes per thread and step, consecutive threads -> consecutive chunks
+#pragma unroll
+        for (int c = 0; c < 8; ++c) sts_zero16B(wr + (c * 128 + r) * 16);
       }
+      TL3_TACC(2)
       ok = ok && mbar_wait(bar_full + 8 * s, ph, wctx, kStDecodeFull);
-      // Residual entries land in any row, so the whole of W_r must be clear before anyone
-      // scatters; the same barrier makes the give-up decision uniform across the group.
+      TL3_TACC(3)
+      // W_r must be clear before anyone scatters into it; the same barrier makes the give-up
+      // decision uniform across the group.
       if (!named_bar_all(1 + g, 128, ok)) break;
+      if (r == 0) TL3_STAMP(i, 2)
       const uint32_t stage = smem_base + static_cast<uint32_t>(s) * a.stage_stride;
       // metadata -> tensor memory (4 columns of this group)
-      {
+      if (!TL3_SKIP(16)) {
         uint32_t m0, m1, m2, m3;
         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(m0), "=r"(m1), "=r"(m2), "=r"(m3) : "r"(stage + kMetaOff + r * 16));
         asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
-                     ::"r"(tmem_base + lane_base + kColMetaT + 4 * g), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
+                     ::"r"(tmem_base + lane_base + kColMetaT + 4 * wb), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
       }
       // byte offset of this thread's chain = exclusive prefix sum of the chain lengths.
       // Each warp scans all 128 lengths (4 per lane) with shuffles; no cross-warp exchange.
@@ -447,9 +521,12 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         off = excl + __dp4a(q & ((1u << (8 * sub)) - 1u), 0x01010101u, 0u);
         len = (q >> (8 * sub)) & 0xFFu;
       }
-      decode_chain(stage, wr, lds_u32(stage + kHdrOff + r * 4), stage + kPddOff + off, len);
+      TL3_TACC(4)
+      if (!TL3_SKIP(4)) decode_chain(stage, wr, lds_u32(stage + kHdrOff + r * 4), stage + kPddOff + off, len);
+      __syncwarp();
+      TL3_TACC(5)
       // Residual layer: (position, value) entries go to W_r too
-      {
+      if (!TL3_SKIP(32)) {
         const uint32_t pdd_len = lds_u32(stage + kInfoOff), res_cnt = lds_u32(stage + kInfoOff + 4);
         const uint32_t res = stage + kPddOff + ((pdd_len + 3u) & ~3u);
         for (uint32_t k = r; k < res_cnt; k += 128) {
@@ -457,73 +534,46 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
           sts_u16(wr + swizzled_offset(rv & 0xFFFFu), rv >> 16);
         }
       }
+      TL3_TACC(6)
       fence_proxy_async_smem();                                   // generic-proxy writes -> MMA reads
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       tc_fence_before();
       mbar_arrive(bar_dec + 8 * s);
-      prev_s = s; prev_ph = ph;
+      if (r == 0) TL3_STAMP(i, 3)
+      TL3_TACC(7)
+#pragma unroll
+      for (int h = kHist - 1; h > 0; --h) { hist_s[h] = hist_s[h - 1]; hist_ph[h] = hist_ph[h - 1]; }
+      hist_s[0] = s; hist_ph[0] = ph;
       s += kGroups;
-      if (s >= S) { s -= S; ph ^= 1u; }
+      while (s >= S) { s -= S; ph ^= 1u; }
     }
+    if (lane == 0) TL3_TDUMP(16 + 8 * (warp - kDecodeWarp0))
   } else if (warp >= kEpilogueWarp0) {
     // ------------------------------------------------------------------ epilogue
     const int et = tid - kEpilogueWarp0 * 32;                    // 0..127 = row of the tile = tensor-memory lane
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     int seg = 0;
     long long t = t_begin;
+    TL3_T0()
     while (t < t_end) {
+      TL3_TACC(0)
       const int mt = static_cast<int>(t / a.tiles_k);
       const long long row_tile_begin = static_cast<long long>(mt) * a.tiles_k, row_tile_end = row_tile_begin + a.tiles_k;
       const long long seg_end = row_tile_end < t_end ? row_tile_end : t_end;
       const bool complete = (t == row_tile_begin) && (seg_end == row_tile_end);
       const int b = seg & 1;
-      if (!named_bar_all(3, 128, mbar_wait(bar_accfull + 8 * b, (seg >> 1) & 1, wctx, kStEpilogueAccFull))) break;
+      if (!named_bar_all(1 + kGroups, 128, mbar_wait(bar_accfull + 8 * b, (seg >> 1) & 1, wctx, kStEpilogueAccFull))) break;
+      TL3_TACC(1)
       tc_fence_after();
-      uint32_t v[NPAD];
-      TmemLd<NPAD>::ld(tmem_base + lane_base + static_cast<uint32_t>(b * NPAD), v);
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      tc_fence_before();
-      mbar_arrive(bar_accempty + 8 * b);
+      constexpr int CH = NPAD < 32 ? NPAD : 32;                 // columns handled per round (register budget)
       const int row = mt * kTileM + et;
-      bool write_y = complete;
-      if (!complete) {
-        // partial sums: slot 2*cta + (this row-tile is not the first one of my range)
-        const int slot = 2 * blockIdx.x + (t_begin < row_tile_begin ? 1 : 0);
-        float* mine = a.partials + static_cast<size_t>(slot) * NPAD * 128 + et;
+      __half* y = a.Y + static_cast<long long>(row) * a.ldy;
+      const bool vec_ok = a.N == NPAD && (a.ldy & 7) == 0 && (reinterpret_cast<uintptr_t>(a.Y) & 15) == 0;
+      auto store_y = [&](const uint32_t* v, int c0) {           // fp32 -> fp16 (round to nearest even) -> Y
+        if (row >= a.M) return;
+        if (vec_ok) {
 #pragma unroll
-        for (int c = 0; c < NPAD; ++c) __stcg(mine + c * 128, __uint_as_float(v[c]));
-        __threadfence();
-        named_bar_sync(3, 128);
-        const int c_first = owner_of(row_tile_begin, T, G), c_last = owner_of(row_tile_end - 1, T, G);
-        if (et == 0) {
-          const unsigned int old = atomicAdd(a.counters + mt, 1u);
-          const bool last = old == static_cast<unsigned int>(c_last - c_first);
-          if (last) a.counters[mt] = 0;                          // leave the workspace cleared
-          *last_flag = last ? 1u : 0u;
-        }
-        named_bar_sync(3, 128);
-        if (*last_flag) {
-          __threadfence();
-          float acc[NPAD];
-#pragma unroll
-          for (int c = 0; c < NPAD; ++c) acc[c] = 0.f;
-          for (int c_id = c_first; c_id <= c_last; ++c_id) {      // fixed order: deterministic sum
-            const int sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
-            const float* p = a.partials + static_cast<size_t>(sl) * NPAD * 128 + et;
-#pragma unroll
-            for (int c = 0; c < NPAD; ++c) acc[c] += __ldcg(p + c * 128);
-          }
-#pragma unroll
-          for (int c = 0; c < NPAD; ++c) v[c] = __float_as_uint(acc[c]);
-          write_y = true;
-        }
-        named_bar_sync(3, 128);                                   // last_flag may be rewritten next segment
-      }
-      if (write_y && row < a.M) {
-        __half* y = a.Y + static_cast<long long>(row) * a.ldy;
-        if (a.N == NPAD && (a.ldy & 7) == 0 && (reinterpret_cast<uintptr_t>(a.Y) & 15) == 0) {
-#pragma unroll
-          for (int c = 0; c < NPAD; c += 8) {
+          for (int c = 0; c < CH; c += 8) {
             uint4 o;
             __half2 h0 = __floats2half2_rn(__uint_as_float(v[c + 0]), __uint_as_float(v[c + 1]));
             __half2 h1 = __floats2half2_rn(__uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
@@ -531,17 +581,69 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
             __half2 h3 = __floats2half2_rn(__uint_as_float(v[c + 6]), __uint_as_float(v[c + 7]));
             o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
             o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
-            *reinterpret_cast<uint4*>(y + c) = o;
+            *reinterpret_cast<uint4*>(y + c0 + c) = o;
           }
         } else {
 #pragma unroll
-          for (int c = 0; c < NPAD; ++c)
-            if (c < a.N) y[c] = __float2half_rn(__uint_as_float(v[c]));
+          for (int c = 0; c < CH; ++c)
+            if (c0 + c < a.N) y[c0 + c] = __float2half_rn(__uint_as_float(v[c]));
+        }
+      };
+      const uint32_t acc_tmem = tmem_base + lane_base + static_cast<uint32_t>(b * NPAD);
+      // partial sums of a shared row-tile: slot 2*cta + (this row-tile is not the first one of my range)
+      const int slot = 2 * blockIdx.x + (t_begin < row_tile_begin ? 1 : 0);
+      float* mine = a.partials + static_cast<size_t>(slot) * NPAD * 128 + et;
+#pragma unroll 1
+      for (int c0 = 0; c0 < NPAD; c0 += CH) {
+        uint32_t v[CH];
+        TmemLd<CH>::ld(acc_tmem + c0, v);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (complete) {
+          store_y(v, c0);
+        } else {
+#pragma unroll
+          for (int c = 0; c < CH; ++c) __stcg(mine + (c0 + c) * 128, __uint_as_float(v[c]));
         }
       }
+      tc_fence_before();
+      mbar_arrive(bar_accempty + 8 * b);
+      if (!complete) {
+        __threadfence();
+        named_bar_sync(1 + kGroups, 128);
+        const int c_first = owner_of(row_tile_begin, T, G), c_last = owner_of(row_tile_end - 1, T, G);
+        if (et == 0) {
+          const unsigned int old = atomicAdd(a.counters + mt, 1u);
+          const bool last = old == static_cast<unsigned int>(c_last - c_first);
+          if (last) a.counters[mt] = 0;                          // leave the workspace cleared
+          *last_flag = last ? 1u : 0u;
+        }
+        named_bar_sync(1 + kGroups, 128);
+        if (*last_flag) {
+          __threadfence();
+#pragma unroll 1
+          for (int c0 = 0; c0 < NPAD; c0 += CH) {
+            float acc[CH];
+#pragma unroll
+            for (int c = 0; c < CH; ++c) acc[c] = 0.f;
+            for (int c_id = c_first; c_id <= c_last; ++c_id) {    // fixed order: deterministic sum
+              const int sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
+              const float* p = a.partials + static_cast<size_t>(sl) * NPAD * 128 + et;
+#pragma unroll
+              for (int c = 0; c < CH; ++c) acc[c] += __ldcg(p + (c0 + c) * 128);
+            }
+            uint32_t v[CH];
+#pragma unroll
+            for (int c = 0; c < CH; ++c) v[c] = __float_as_uint(acc[c]);
+            store_y(v, c0);
+          }
+        }
+        named_bar_sync(1 + kGroups, 128);                         // last_flag may be rewritten next segment
+      }
+      TL3_TACC(2)
       ++seg;
       t = seg_end;
     }
+    if (et == 0) TL3_TDUMP(160)
   }
 
   // ------------------------------------------------------------------ teardown
@@ -677,7 +779,7 @@ int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t l
   const uint32_t block_area = (m->max_block_bytes + 16u + 1023u) / 1024u * 1024u;
   const uint32_t x_bytes = 128u * n_pad * 2u;
   const uint32_t stage_stride = block_area + x_bytes;
-  const uint32_t fixed = kGroups * kWrBytes + kBarrierBytes + 1024u;   // + alignment slack
+  const uint32_t fixed = kWrBuffers * kWrBytes + kBarrierBytes + 1024u;   // + alignment slack
   if (fixed + 2u * stage_stride > kSmemLimit) return TL3_ERR_UNSUPPORTED;
   int stages = static_cast<int>((kSmemLimit - fixed) / stage_stride);
   if (stages > kMaxStages) stages = kMaxStages;
@@ -716,6 +818,13 @@ int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t l
   args.stage_stride = stage_stride;
   args.x_offset = block_area;
   args.num_stages = stages;
+#ifdef TL3_PHASE_TIMING
+  args.timing = g_timing_buffer;
+  args.debug_skip = getenv("TL3_DEBUG_SKIP") ? atoi(getenv("TL3_DEBUG_SKIP")) : 0;
+#else
+  args.timing = nullptr;
+  args.debug_skip = 0;
+#endif
   m->last_ctas = grid; m->last_stages = stages; m->last_smem = static_cast<int>(smem_bytes);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   switch (n_pad) {
@@ -757,5 +866,9 @@ int tl3_last_launch(const tl3_matrix* m, int* ctas, int* stages, int* smem_bytes
 }
 
 int tl3_last_cuda_error(void) { return tl3::g_last_cuda_error; }
+
+#ifdef TL3_PHASE_TIMING
+void tl3_debug_set_timing_buffer(long long* device_ptr) { tl3::g_timing_buffer = device_ptr; }
+#endif
 
 }  // extern "C"
