@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of the three-layer sparse SpMM on B200.
+
+One "step" = one pass of the whole hot path over the OPT-13B-shaped workload (configs[1] of
+the benchmark spec): W of 5120x5120, 20480x5120 and 5120x20480 at 50 % per-row magnitude sparsity,
+each multiplied by X with N = 8, 16 and 32 -- nine SpMM launches on one stream.  The order is
+N-major, so 297 MB of other weights stream through the 126 MB L2 between two uses of a matrix.
+
+Prints ONE JSON line (rank 0).  `value` is the achieved HBM rate: algorithmic bytes of a step
+(compressed W blob + X + Y of every launch) / device time of the step, inputs resident in HBM.
+`e2e` is the same metric through tl3_spmm_host (host X and Y, copies inside the timed region).
+
+`--impl reference` times the CPU oracle (oracle/, unmodified) on the same metric and workload,
+on a bounded sample per step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2607_08786_b200 import dist, workloads as wl  # noqa: E402
+
+METRIC = "spmm_achieved_hbm_gbs"
+UNIT = "GB/s"
+WORKLOAD = "config2_opt13b_shapes_50pct_N8_16_32"
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch / its algorithmic bytes, from the
+# ncu capture summarised in profiles/tl3_spmm_kernel_8192x8192_n16.md (scaled by bytes, since
+# traffic grows in proportion to the blob)
+NCU_TRAFFIC_RATIO = 1.05
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def measured_peak_gbs():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+def step_cases(seed_offset: int = 0):
+    """Config 2 in launch order: N-major, shapes inside."""
+    cases = list(wl.config_cases(2))
+    out = []
+    for N in (8, 16, 32):
+        for c in cases:
+            if c.N == N:
+                out.append(wl.Case(c.config, c.name, c.M, c.K, c.N, c.seed + seed_offset, c.sparsity, c.kind))
+    return out
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except Exception:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+def run_reference(args, rank):
+    """CPU oracle on the host cores: same metric, bounded sample of the same workload per step."""
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    sample = [c for c in step_cases() if c.N == 16 and c.M == 5120 and c.K == 5120]   # one matrix, N = 16
+    prepared = []
+    for c in sample:
+        W, X = c.make_W(), c.make_X()
+        cont = oracle.encode(W)
+        prepared.append((cont, X, cont.nbytes() + X.nbytes + c.M * c.N * 2))
+    def step():
+        for cont, X, _ in prepared:
+            oracle.spmm(cont, X)
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    nbytes = sum(b for _, _, b in prepared)
+    value = nbytes / dt / 1e9
+    desc = {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": "5120x5120 at N=16 (1 of the 9 launches of a step), canonical container bytes"}
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": desc["sample"]},
+        "cpu_baseline": desc,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+def run_ours(args, rank, local_rank, world):
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    from paper_2607_08786_b200 import build, tl3
+    build.build_library()
+    tl3.lib()
+    dev = torch.device("cuda", local_rank)
+
+    cases = step_cases(dist.rank_seed_offset(rank))
+    mats, dense = {}, {}
+    launches = []
+    t_setup = time.time()
+    for c in cases:
+        key = (c.M, c.K)
+        if key not in mats:
+            W = c.make_W()
+            m = tl3.encode(W)
+            m.upload(device=dev)
+            mats[key] = m
+            dense[key] = torch.from_numpy(W).to(dev)
+            st = m.stats()
+            log(f"[rank {rank}] {c.M}x{c.K}: nnz {st['nnz']} TC {st['n_tc']/st['nnz']:.4f} SF {st['n_sf']/st['nnz']:.4f} "
+                f"RES {st['n_res']/st['nnz']:.4f} dummies {st['n_dummy']/st['nnz']:.4f} blob {st['device_bytes']/1e6:.1f} MB "
+                f"({st['device_bytes']/(2*c.M*c.K):.4f} x dense, canonical {st['canonical_bytes']/(2*c.M*c.K):.4f})")
+        m = mats[key]
+        X = c.make_X()
+        Xd = torch.from_numpy(X).to(dev)
+        Y = torch.empty((c.M, c.N), dtype=torch.float16, device=dev)
+        ws = m.new_workspace(c.N)
+        nbytes = m.device_bytes() + X.nbytes + c.M * c.N * 2
+        launches.append(dict(case=c, m=m, X=Xd, Y=Y, ws=ws, bytes=nbytes, Xh=X, flops=2.0 * c.M * c.K * c.N))
+    torch.cuda.synchronize()
+    log(f"[rank {rank}] setup {time.time() - t_setup:.1f} s")
+
+    stream = torch.cuda.current_stream()
+
+    def step_eager():
+        for L in launches:
+            L["m"].spmm(L["X"], L["Y"], workspace=L["ws"])
+
+    # the nine launches as one CUDA graph (removes host launch gaps); eager if capture is refused
+    graph = None
+    try:
+        step_eager()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            step_eager()
+        graph = g
+    except Exception as e:  # pragma: no cover
+        log(f"[rank {rank}] CUDA graph capture failed ({e}); timing eager launches")
+        graph = None
+    step = graph.replay if graph is not None else step_eager
+    stream = torch.cuda.current_stream()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    for L in launches:
+        assert L["m"].status(L["ws"]) == tl3.OK
+
+    # ---- timed region: exactly K steps, device time, max over ranks
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    dist.barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    ms_total = dist.max_over_ranks(ms_total, device=dev)
+    ms_step = ms_total / args.steps
+    step_bytes = sum(L["bytes"] for L in launches)
+    total_bytes = dist.sum_over_ranks(step_bytes, device=dev)
+    value = total_bytes / (ms_step * 1e-3) / 1e9
+
+    # ---- per-launch kernel durations (CUDA events around each launch, same stream, same order)
+    per = [[] for _ in launches]
+    reps = max(3, min(args.steps, 10))
+    for _ in range(reps):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(launches) + 1)]
+        evs[0].record(stream)
+        for i, L in enumerate(launches):
+            L["m"].spmm(L["X"], L["Y"], workspace=L["ws"])
+            evs[i + 1].record(stream)
+        torch.cuda.synchronize()
+        for i in range(len(launches)):
+            per[i].append(evs[i].elapsed_time(evs[i + 1]) * 1e3)
+    us = [float(np.median(p)) for p in per]
+
+    # ---- same-shape dense fp16 GEMM (cuBLAS through torch.matmul), same order, same protocol
+    dper = [[] for _ in launches]
+    outs = [torch.empty((L["case"].M, L["case"].N), dtype=torch.float16, device=dev) for L in launches]
+    for rep in range(reps + 2):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(launches) + 1)]
+        evs[0].record(stream)
+        for i, L in enumerate(launches):
+            torch.matmul(dense[(L["case"].M, L["case"].K)], L["X"], out=outs[i])
+            evs[i + 1].record(stream)
+        torch.cuda.synchronize()
+        if rep >= 2:
+            for i in range(len(launches)):
+                dper[i].append(evs[i].elapsed_time(evs[i + 1]) * 1e3)
+    dus = [float(np.median(p)) for p in dper]
+
+    # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region
+    e2e_bufs = []
+    for L in launches:
+        c = L["case"]
+        Xp = torch.from_numpy(L["Xh"]).pin_memory()
+        Yp = torch.empty((c.M, c.N), dtype=torch.float16).pin_memory()
+        dX = torch.empty(c.K * ((c.N + 7) // 8 * 8) * 2, dtype=torch.uint8, device=dev)
+        dY = torch.empty(c.M * c.N * 2, dtype=torch.uint8, device=dev)
+        e2e_bufs.append((Xp.numpy(), Yp.numpy(), dX, dY))
+
+    def step_e2e():
+        for L, (Xp, Yp, dX, dY) in zip(launches, e2e_bufs):
+            L["m"].spmm_host(Xp, Yp, dX, dY, L["ws"])
+
+    for _ in range(3):
+        step_e2e()
+    dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step_e2e()
+    torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / args.steps
+    e2e_s = dist.max_over_ranks(e2e_s, device=dev)
+    e2e_value = total_bytes / e2e_s / 1e9
+    h2d = sum(L["Xh"].nbytes for L in launches)
+    d2h = sum(L["case"].M * L["case"].N * 2 for L in launches)
+    # the host-buffer path must give the same numbers as the device path
+    for L, (Xp, Yp, dX, dY) in zip(launches[:2], e2e_bufs[:2]):
+        assert np.array_equal(Yp.view(np.uint16), L["Y"].cpu().numpy().view(np.uint16))
+
+    if rank != 0:
+        return
+
+    # ---- CPU baseline: the oracle as it stands on a bounded sample (rank 0, N = 1 only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        c = [x for x in cases if x.M == 5120 and x.K == 5120 and x.N == 16][0]
+        W, X = c.make_W(), c.make_X()
+        cont = oracle.encode(W)
+        oracle.spmm(cont, X)
+        ts = []
+        for _ in range(3):
+            t0 = time.perf_counter()
+            Yo = oracle.spmm(cont, X)
+            ts.append(time.perf_counter() - t0)
+        nb = cont.nbytes() + X.nbytes + c.M * c.N * 2
+        cpu = {"value": nb / min(ts) / 1e9, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+               "sample": "5120x5120 at N=16 (1 of the 9 launches of a step), best of 3",
+               "us": min(ts) * 1e6}
+        # and the parity of that launch, while the oracle's result is at hand
+        Yg = [L for L in launches if L["case"] is c][0]["Y"].cpu().numpy().astype(np.float64)
+        Yref, bound = oracle.dense_fp64(W, X)
+        assert np.all(np.abs(Yg - Yref) <= oracle.tolerance(bound)), "GPU result outside tolerance"
+        assert np.all(np.abs(Yo.view(np.float16).astype(np.float64) - Yref) <= oracle.tolerance(bound))
+
+    peak, peak_kind = measured_peak_gbs()
+    kern_s = sum(us) * 1e-6
+    achieved = step_bytes / kern_s / 1e9
+    table = []
+    for L, u, du in zip(launches, us, dus):
+        c = L["case"]
+        table.append({"M": c.M, "K": c.K, "N": c.N, "us": round(u, 2), "gbs": round(L["bytes"] / u / 1e3, 1),
+                      "frac_measured": round(L["bytes"] / u / 1e3 / peak, 4),
+                      "frac_nominal_8tbs": round(L["bytes"] / u / 1e3 / 8000.0, 4),
+                      "dense_equiv_tflops": round(L["flops"] / u / 1e6, 2),
+                      "dense_gemm_us": round(du, 2), "speedup_vs_dense": round(du / u, 3)})
+    ll = launches[0]["m"].last_launch()
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f16xf16->f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "launches_per_step": len(launches), "order": "N-major",
+                   "l2": "inputs larger than L2: 297 MB of other weights stream between two uses of a matrix",
+                   "bytes_per_step": step_bytes, "graph": graph is not None,
+                   "ctas": ll["ctas"], "smem_bytes": ll["smem_bytes"]},
+        "clocks": clocks,
+        "gpu_launches": len(launches) * args.steps,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_s * 1e3},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "frac_nominal_8tbs": achieved / 8000.0,
+                     "traffic": NCU_TRAFFIC_RATIO * step_bytes / len(launches),
+                     "kernel": "tl3_spmm_kernel", "kernel_us_per_step": sum(us),
+                     "algorithmic_bytes_per_launch": step_bytes / len(launches)},
+        "cpu_baseline": cpu,
+        "dense_fp16_gemm": {"us_per_step": sum(dus), "speedup_of_spmm": sum(dus) / sum(us)},
+        "per_launch": table,
+    }
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank, local_rank, world = dist.env_world()
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if world > 1:
+        dist.init_process_group("nccl")
+    run_ours(args, rank, local_rank, world)
+    if world > 1:
+        import torch.distributed as td
+        td.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

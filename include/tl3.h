@@ -100,6 +100,13 @@ void tl3_free(tl3_matrix* m);
 /* Size of the packed device blob (tile blocks ready for bulk copies). */
 size_t tl3_device_bytes(const tl3_matrix* m);
 
+/* Pack the container into a HOST buffer of tl3_device_bytes() bytes: exactly the bytes tl3_upload()
+ * sends to the device (a permutation of the canonical arrays plus alignment padding: per tile one
+ * contiguous block holding the value slots in the shared-memory image the MMA reads, the metadata
+ * in tensor-memory word order, the chain starts, lengths and delta bytes, and the Residual
+ * entries).  For callers that stage the blob themselves.  Errors: UNSUPPORTED, INVALID_ARG. */
+int tl3_pack(const tl3_matrix* m, void* host_buf, size_t bytes);
+
 /* Pack the container and copy it to dptr (device, >= tl3_device_bytes(), 256-byte aligned) on
  * `stream` (a cudaStream_t passed as void*; NULL = default stream), then bind dptr to the handle.
  * The copy is asynchronous with respect to the device; host staging is released before return.

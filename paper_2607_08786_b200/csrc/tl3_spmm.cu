@@ -731,6 +731,14 @@ size_t tl3_device_bytes(const tl3_matrix* m) {
   return tl3::plan_device_layout(const_cast<tl3_matrix*>(m));
 }
 
+int tl3_pack(const tl3_matrix* m, void* host_buf, size_t bytes) {
+  if (!m || !host_buf) return TL3_ERR_INVALID_ARG;
+  if (m->p.tile_m != tl3::kTileM || m->p.tile_k != tl3::kTileK) return TL3_ERR_UNSUPPORTED;
+  if (bytes < tl3::plan_device_layout(const_cast<tl3_matrix*>(m))) return TL3_ERR_INVALID_ARG;
+  tl3::pack_device_blob(m, static_cast<uint8_t*>(host_buf));
+  return TL3_OK;
+}
+
 int tl3_upload(tl3_matrix* m, void* dptr, void* stream) {
   if (!m || !dptr || (reinterpret_cast<uintptr_t>(dptr) & 255) != 0) return TL3_ERR_INVALID_ARG;
   if (m->p.tile_m != tl3::kTileM || m->p.tile_k != tl3::kTileK) return TL3_ERR_UNSUPPORTED;

@@ -25,7 +25,7 @@ _CANONICAL_DTYPES = (np.uint16, np.uint8, np.uint16, np.uint16, np.uint8, np.uin
 
 # every symbol include/tl3.h declares
 SYMBOLS = ("tl3_encode", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_deserialize",
-           "tl3_free", "tl3_device_bytes", "tl3_upload", "tl3_workspace_bytes", "tl3_workspace_init",
+           "tl3_free", "tl3_device_bytes", "tl3_pack", "tl3_upload", "tl3_workspace_bytes", "tl3_workspace_init",
            "tl3_spmm", "tl3_spmm_host", "tl3_status", "tl3_last_launch", "tl3_strerror",
            "tl3_last_cuda_error")
 
@@ -74,6 +74,7 @@ def lib() -> ctypes.CDLL:
         L.tl3_free.restype = None
         L.tl3_device_bytes.argtypes = [vp]
         L.tl3_device_bytes.restype = sz
+        L.tl3_pack.argtypes = [vp, vp, sz]
         L.tl3_upload.argtypes = [vp, vp, vp]
         L.tl3_workspace_bytes.argtypes = [vp, ci]
         L.tl3_workspace_bytes.restype = sz
@@ -190,6 +191,12 @@ class Matrix:
     # -- device side -------------------------------------------------------------------------
     def device_bytes(self) -> int:
         return int(lib().tl3_device_bytes(self._h))
+
+    def pack(self) -> np.ndarray:
+        """The device blob as a host uint8 array (what ``upload`` copies to the GPU)."""
+        buf = np.empty(self.device_bytes(), dtype=np.uint8)
+        _check(lib().tl3_pack(self._h, buf.ctypes.data, buf.nbytes), "tl3_pack")
+        return buf
 
     def upload(self, device="cuda", stream=None):
         """Allocates the blob as a torch.uint8 tensor, packs and copies the matrix into it."""

@@ -1,0 +1,236 @@
+"""Parity of the CUDA SpMM with the CPU oracle (needs a B200).  Everything goes through the C ABI.
+
+Y is compared element by element with the dense float64 product of the masked W (the plain
+definition), within the tolerance of the benchmark spec, |y - y_ref| <= 2e-3 * sum_k |w_ik x_kj|
++ 1e-3, and with the oracle's own format-walking SpMM.  Cases where all partial sums are exactly
+representable (identity X, small integers) must match bit for bit.
+"""
+import numpy as np
+import pytest
+
+from paper_2607_08786_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def tl3():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2607_08786_b200 import build, tl3 as mod
+    build.build_library()
+    mod.lib()                                   # raises if the CUDA library is missing: no fallback
+    return mod
+
+
+def device_X(X, ld=None):
+    import torch
+    K, N = X.shape
+    ld = ld or (N + 7) // 8 * 8
+    buf = torch.zeros((K, ld), dtype=torch.float16, device="cuda")
+    buf[:, :N] = torch.from_numpy(X)
+    return buf[:, :N]
+
+
+def run_gpu(tl3, W, X, ldx=None, ldy=None, repeats=1):
+    import torch
+    m = tl3.encode(W)
+    m.upload()
+    Xd = device_X(X, ldx)
+    N = X.shape[1]
+    ws = m.new_workspace(N)
+    Ybuf = torch.full((W.shape[0], ldy or N), float("nan"), dtype=torch.float16, device="cuda")
+    Y = Ybuf[:, :N]
+    outs = []
+    for _ in range(repeats):
+        m.spmm(Xd, Y, workspace=ws)
+        torch.cuda.synchronize()
+        assert m.status(ws) == tl3.OK
+        outs.append(Y.cpu().numpy().copy())
+    if ldy and ldy > N:                          # columns beyond N are left alone
+        assert torch.isnan(Ybuf[:, N:]).all()
+    for o in outs[1:]:
+        assert np.array_equal(o.view(np.uint16), outs[0].view(np.uint16))   # deterministic
+    return outs[0], m
+
+
+def check(oracle_mod, W, X, Y, with_oracle_spmm=True):
+    Yref, bound = oracle_mod.dense_fp64(W, X)
+    err = np.abs(Y.astype(np.float64) - Yref)
+    tol = oracle_mod.tolerance(bound)
+    assert np.all(err <= tol), f"max err/tol {np.max(err / tol):.3f} at {np.unravel_index(np.argmax(err / tol), err.shape)}"
+    if with_oracle_spmm:
+        Yo = oracle_mod.spmm(oracle_mod.encode(W), X).view(np.float16).astype(np.float64)
+        # both accumulate in fp32 (different order) and round once to fp16
+        assert np.all(np.abs(Y.astype(np.float64) - Yo) <= 2.0**-9 * np.abs(Yo) + 1e-4 * bound + 1e-6)
+
+
+def test_config1(tl3, oracle_mod):
+    case = next(wl.config_cases(1))
+    W, X = case.make_W(), case.make_X()
+    Y, m = run_gpu(tl3, W, X, repeats=3)
+    check(oracle_mod, W, X, Y)
+    assert m.last_launch()["ctas"] == 64
+
+
+@pytest.mark.parametrize("N", [1, 5, 8, 16, 24, 32, 48, 64])
+def test_all_widths(tl3, oracle_mod, N):
+    case = wl.Case(0, "n", 640, 896, N, 40 + N, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    Y, _ = run_gpu(tl3, W, X, repeats=2)
+    check(oracle_mod, W, X, Y)
+
+
+@pytest.mark.parametrize("shape", [(1, 8), (127, 129), (130, 260), (1000, 1096), (384, 128), (128, 4096), (4096, 128)])
+def test_ragged_shapes(tl3, oracle_mod, shape):
+    case = wl.Case(0, "r", shape[0], shape[1], 16, shape[0] + shape[1], 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    Y, _ = run_gpu(tl3, W, X)
+    check(oracle_mod, W, X, Y)
+
+
+@pytest.mark.parametrize("sparsity,kind", [(0.4, "magnitude"), (0.6, "magnitude"), (0.7, "magnitude"),
+                                           (0.5, "wanda"), (0.5, "row_scaled"), (0.5, "bernoulli")])
+def test_sparsities_and_masks(tl3, oracle_mod, sparsity, kind):
+    case = wl.Case(0, "s", 1536, 2048, 16, int(sparsity * 100), sparsity, kind)
+    W, X = case.make_W(), case.make_X()
+    Y, _ = run_gpu(tl3, W, X)
+    check(oracle_mod, W, X, Y)
+
+
+def test_split_k_many_and_few_contributors(tl3, oracle_mod):
+    # 2 row-tiles x 160 k-tiles: every row-tile is shared by ~74 CTAs
+    case = wl.Case(0, "wide", 256, 20480, 8, 77, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    Y, m = run_gpu(tl3, W, X, repeats=2)
+    check(oracle_mod, W, X, Y)
+    assert m.last_launch()["ctas"] == 148
+    # 160 row-tiles x 2 k-tiles: most row-tiles belong to one CTA, some straddle two
+    case = wl.Case(0, "tall", 20480, 256, 8, 78, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    Y, _ = run_gpu(tl3, W, X, repeats=2)
+    check(oracle_mod, W, X, Y)
+
+
+def test_degenerate_matrices(tl3, oracle_mod):
+    rng = np.random.default_rng(3)
+    X = rng.standard_normal((512, 16)).astype(np.float16)
+    Z = np.zeros((256, 512), dtype=np.float16)
+    Y, _ = run_gpu(tl3, Z, X)
+    assert not Y.view(np.uint16).any()                             # all-zero W: exact zeros
+    D = (rng.standard_normal((256, 512)) * 0.05).astype(np.float16)   # fully dense: half of nnz is Residual
+    D[D == 0] = np.float16(0.01)
+    Y, m = run_gpu(tl3, D, X)
+    assert m.stats()["n_res"] == D.size // 2
+    check(oracle_mod, D, X, Y)
+    keep = np.zeros((256, 128, 4), dtype=bool)                        # exact 2:4: only the Sparse-TC layer
+    keep[:, :, [0, 3]] = True
+    W24 = np.where(keep.reshape(256, 512), D, np.float16(0))
+    Y, m = run_gpu(tl3, W24, X)
+    assert m.stats()["n_sf"] == 0 and m.stats()["n_res"] == 0
+    check(oracle_mod, W24, X, Y)
+    T = np.zeros((256, 512), dtype=np.float16)                        # every surplus parked in another row
+    T[:64] = D[:64]
+    T[128:192] = D[128:192]
+    Y, _ = run_gpu(tl3, T, X)
+    check(oracle_mod, T, X, Y)
+
+
+def test_identity_X_reproduces_W_bit_for_bit(tl3):
+    """Each y_ij is one product w_ij * 1: the GPU must hand back the decoded W exactly."""
+    for k0 in (0, 64):
+        case = wl.Case(0, "id", 512, 128, 64, 90 + k0, 0.5, "magnitude")
+        W = case.make_W()
+        X = np.zeros((128, 64), dtype=np.float16)
+        X[k0:k0 + 64] = np.eye(64, dtype=np.float16)
+        Y, _ = run_gpu(tl3, W, X)
+        assert np.array_equal(Y.view(np.uint16), W[:, k0:k0 + 64].view(np.uint16))
+
+
+def test_small_integers_are_exact(tl3, oracle_mod):
+    rng = np.random.default_rng(12)
+    W = np.where(rng.random((384, 1280)) < 0.5, rng.integers(-4, 5, (384, 1280)), 0).astype(np.float16)
+    X = rng.integers(-3, 4, (1280, 32)).astype(np.float16)
+    Y, _ = run_gpu(tl3, W, X)
+    assert np.array_equal(Y.astype(np.int64), W.astype(np.int64) @ X.astype(np.int64))
+    assert np.array_equal(Y.view(np.uint16), oracle_mod.spmm(oracle_mod.encode(W), X))
+
+
+def test_strided_operands(tl3, oracle_mod):
+    case = wl.Case(0, "ld", 300, 700, 12, 5, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    Y, _ = run_gpu(tl3, W, X, ldx=40, ldy=19)
+    check(oracle_mod, W, X, Y)
+
+
+def test_argument_errors_on_device(tl3):
+    import torch
+    case = wl.Case(0, "e", 256, 256, 8, 5, 0.5, "magnitude")
+    m = tl3.encode(case.make_W())
+    X = torch.zeros((256, 8), dtype=torch.float16, device="cuda")
+    Y = torch.zeros((256, 8), dtype=torch.float16, device="cuda")
+    L = tl3.lib()
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    assert L.tl3_spmm(m._h, X.data_ptr(), 8, Y.data_ptr(), 8, 8, ws.data_ptr(), None) == tl3.ERR_NOT_UPLOADED
+    m.upload()
+    ws = m.new_workspace(8)
+    assert L.tl3_spmm(m._h, X.data_ptr(), 8, Y.data_ptr(), 8, 65, ws.data_ptr(), None) == tl3.ERR_UNSUPPORTED
+    assert L.tl3_spmm(m._h, X.data_ptr(), 8, Y.data_ptr(), 8, 0, ws.data_ptr(), None) == tl3.ERR_UNSUPPORTED
+    assert L.tl3_spmm(m._h, X.data_ptr(), 12, Y.data_ptr(), 8, 8, ws.data_ptr(), None) == tl3.ERR_INVALID_ARG   # ldx % 8
+    assert L.tl3_spmm(m._h, X.data_ptr() + 2, 8, Y.data_ptr(), 8, 8, ws.data_ptr(), None) == tl3.ERR_INVALID_ARG  # X alignment
+    assert L.tl3_spmm(m._h, X.data_ptr(), 8, Y.data_ptr(), 4, 8, ws.data_ptr(), None) == tl3.ERR_INVALID_ARG    # ldy < N
+    assert L.tl3_spmm(m._h, X.data_ptr(), 8, Y.data_ptr(), 8, 8, ws.data_ptr(), None) == tl3.OK
+    torch.cuda.synchronize()
+    assert m.status(ws) == tl3.OK
+
+
+def test_host_buffer_entry_point(tl3, oracle_mod):
+    import torch
+    case = wl.Case(0, "h", 640, 512, 12, 8, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    m = tl3.encode(W)
+    m.upload()
+    ws = m.new_workspace(case.N)
+    dX = torch.empty(case.K * 16 * 2, dtype=torch.uint8, device="cuda")
+    dY = torch.empty(case.M * case.N * 2, dtype=torch.uint8, device="cuda")
+    Y = np.zeros((case.M, case.N), dtype=np.float16)
+    m.spmm_host(X, Y, dX, dY, ws)
+    check(oracle_mod, W, X, Y)
+
+
+def _sampled_check(oracle_mod, W, X, Y, rows):
+    Yref, bound = oracle_mod.dense_fp64(W[rows], X)
+    err = np.abs(Y[rows].astype(np.float64) - Yref)
+    assert np.all(err <= oracle_mod.tolerance(bound))
+
+
+@pytest.mark.parametrize("config", [2, 3, 4, 5])
+def test_full_size_configs_sampled(tl3, oracle_mod, config):
+    """The benchmark's shapes in the benchmark's launch configuration; the float64 definition is
+    evaluated on a sample of rows (all columns) that covers first, last and straddling row-tiles."""
+    import torch
+    seen = set()
+    for case in wl.config_cases(config):
+        key = (case.M, case.K, case.seed)
+        if config == 4 and case.M * case.K > 100e6 and case.N != 64:
+            continue                                         # the two largest shapes once, at the widest N
+        W = case.make_W()
+        m = tl3.encode(W)
+        if key not in seen:
+            seen.add(key)
+            assert np.array_equal(m.decode(), W.view(np.uint16))       # bit-exact round trip at full size
+        m.upload()
+        Xd = torch.from_numpy(case.make_X()).cuda()
+        ws = m.new_workspace(case.N)
+        Y = m.spmm(Xd, workspace=ws)
+        torch.cuda.synchronize()
+        assert m.status(ws) == tl3.OK
+        Yh = Y.cpu().numpy()
+        rng = np.random.default_rng(case.seed)
+        rows = np.unique(np.concatenate([np.arange(0, 130), np.arange(case.M - 130, case.M),
+                                         rng.integers(0, case.M, 700)]))
+        _sampled_check(oracle_mod, W, Xd.cpu().numpy(), Yh, rows)
+        assert np.isfinite(Yh.astype(np.float32)).all()
+        m.close()
+        del Xd, Y, ws
+        torch.cuda.empty_cache()
