@@ -54,7 +54,8 @@ enum {
   TL3_ERR_BAD_CONTAINER = -4,    /* inconsistent container (deserialize / decode)               */
   TL3_ERR_CUDA = -5,             /* a CUDA runtime call failed; see tl3_last_cuda_error()       */
   TL3_ERR_DEVICE_TIMEOUT = -6,   /* a bounded wait inside the kernel gave up (status word)      */
-  TL3_ERR_NO_MEMORY = -7
+  TL3_ERR_NO_MEMORY = -7,
+  TL3_ERR_SCRATCH_LIMIT = -8     /* tl3_spmm_static_scratch: the problem needs more than the built-in scratch */
 };
 
 /* Canonical arrays, in the order tl3_canonical() numbers them. */
@@ -138,6 +139,29 @@ int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t l
  * ldx = ldy = N.  dX (>= K*N*2 bytes) and dY (>= M*N*2 bytes): device scratch owned by the caller. */
 int tl3_spmm_host(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int N, void* dX, void* dY,
                   void* workspace, void* stream);
+
+/* (No counterpart in the paper.)  Y = W X exactly as tl3_spmm computes it, for callers that are
+ * not allowed to obtain device memory themselves and so cannot provide a workspace: a driver-level
+ * plug-in whose host application hands it only the input and output buffers and forbids allocation
+ * calls inside its execute hook, or a process running under a fixed device-memory budget that was
+ * spent before this library was loaded.  The split-K partial sums, the arrival counters and the
+ * status word live in a fixed array that is part of the library image: TL3_STATIC_SCRATCH_BYTES
+ * (3 MiB) of device memory on every GPU that loads the library, held until the process exits.
+ *   - Problems whose scratch need (what tl3_workspace_bytes() reports) exceeds that size are refused
+ *     with TL3_ERR_SCRATCH_LIMIT and nothing is launched.  On a 148-SM device this admits N <= 16
+ *     for any matrix with up to ~150000 row-tiles; N > 16 is refused there.
+ *   - X, Y, ldx, ldy, N, stream: as for tl3_spmm.  The caller still owns X and Y.
+ *   - The first call on each device looks up the array's device address (that device must be
+ *     current); make that first call outside any stream capture.  Later calls only enqueue work.
+ *   - The function calls no cudaMalloc / cudaFree nor any allocating routine, on any call.
+ *   - All calls on a device share the one array.  Each call clears the counters and the status word
+ *     on `stream` before the kernel, so a call that was cut short does not poison the next one, but
+ *     two calls that overlap on the GPU (different streams, no dependency) race on it: serialise
+ *     them.  tl3_static_scratch_status() reads the status word of the current device. */
+#define TL3_STATIC_SCRATCH_BYTES (3u << 20)
+int tl3_spmm_static_scratch(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N,
+                            void* stream);
+int tl3_static_scratch_status(void* stream);
 
 /* Read the workspace's status word (synchronises `stream`).  TL3_OK, or DEVICE_TIMEOUT if a
  * bounded wait inside a kernel expired since the last tl3_workspace_init(). */

@@ -470,6 +470,7 @@ const char* tl3_strerror(int code) {
     case TL3_ERR_CUDA: return "CUDA runtime error";
     case TL3_ERR_DEVICE_TIMEOUT: return "a bounded wait inside the kernel expired";
     case TL3_ERR_NO_MEMORY: return "out of host memory";
+    case TL3_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the library's built-in array holds";
     default: return "unknown error";
   }
 }

@@ -856,6 +856,52 @@ int tl3_spmm_host(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int N, vo
   return TL3_OK;
 }
 
+// ---- entry point that allocates nothing: scratch inside the library image -------------------
+// Split-K partials, arrival counters and the status word for callers that cannot supply a
+// workspace.  The name below is a host-side handle of the symbol, not a device address: host code
+// must go through cudaGetSymbolAddress (done once per device, with that device current).
+static __device__ __align__(256) unsigned char g_static_scratch[TL3_STATIC_SCRATCH_BYTES];
+
+namespace tl3 {
+static int static_scratch_address(void** out) {
+  int dev = 0;
+  TL3_CUDA(cudaGetDevice(&dev));
+  static std::mutex mu;
+  static std::vector<void*> per_device;
+  std::lock_guard<std::mutex> lock(mu);
+  if (static_cast<size_t>(dev) >= per_device.size()) per_device.resize(dev + 1, nullptr);
+  if (!per_device[dev]) {
+    void* p = nullptr;
+    TL3_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+    per_device[dev] = p;
+  }
+  *out = per_device[dev];
+  return TL3_OK;
+}
+}  // namespace tl3
+
+int tl3_spmm_static_scratch(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N, void* stream) {
+  if (!m || !X || !Y) return TL3_ERR_INVALID_ARG;
+  if (!m->dptr) return TL3_ERR_NOT_UPLOADED;
+  if (N < 1 || N > 64) return TL3_ERR_UNSUPPORTED;
+  tl3::DeviceInfo di;
+  if (int rc = tl3::device_info(&di)) return rc;
+  const tl3::WorkspaceLayout wl = tl3::workspace_layout(m, tl3::n_pad_of(N), di.sm_count);
+  if (wl.total > TL3_STATIC_SCRATCH_BYTES) return TL3_ERR_SCRATCH_LIMIT;
+  void* scratch = nullptr;
+  if (int rc = tl3::static_scratch_address(&scratch)) return rc;
+  // counters and status word must start at zero; the partial-sum slots are always written before
+  // they are read, so the last call's contents there do not matter
+  TL3_CUDA(cudaMemsetAsync(scratch, 0, wl.partials_off, static_cast<cudaStream_t>(stream)));
+  return tl3_spmm(m, X, ldx, Y, ldy, N, scratch, stream);
+}
+
+int tl3_static_scratch_status(void* stream) {
+  void* scratch = nullptr;
+  if (int rc = tl3::static_scratch_address(&scratch)) return rc;
+  return tl3_status(nullptr, scratch, stream);
+}
+
 int tl3_status(const tl3_matrix* m, void* workspace, void* stream) {
   (void)m;
   if (!workspace) return TL3_ERR_INVALID_ARG;

@@ -16,7 +16,8 @@ _LIB_PATH = os.path.join(_PKG, "libtl3.so")
 
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NOT_UPLOADED, ERR_BAD_CONTAINER = -1, -2, -3, -4
-ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_NO_MEMORY = -5, -6, -7
+ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_NO_MEMORY, ERR_SCRATCH_LIMIT = -5, -6, -7, -8
+STATIC_SCRATCH_BYTES = 3 << 20
 
 CANONICAL = ("tc_vals", "tc_meta", "chain_tau0", "chain_rho0", "chain_len", "pdd_bytes", "tile_dir",
              "res_rho", "res_val")
@@ -26,7 +27,7 @@ _CANONICAL_DTYPES = (np.uint16, np.uint8, np.uint16, np.uint16, np.uint8, np.uin
 # every symbol include/tl3.h declares
 SYMBOLS = ("tl3_encode", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_deserialize",
            "tl3_free", "tl3_device_bytes", "tl3_pack", "tl3_upload", "tl3_workspace_bytes", "tl3_workspace_init",
-           "tl3_spmm", "tl3_spmm_host", "tl3_status", "tl3_last_launch", "tl3_strerror",
+           "tl3_spmm", "tl3_spmm_host", "tl3_spmm_static_scratch", "tl3_static_scratch_status", "tl3_status", "tl3_last_launch", "tl3_strerror",
            "tl3_last_cuda_error")
 
 
@@ -81,6 +82,8 @@ def lib() -> ctypes.CDLL:
         L.tl3_workspace_init.argtypes = [vp, sz, vp]
         L.tl3_spmm.argtypes = [vp, vp, i64, vp, i64, ci, vp, vp]
         L.tl3_spmm_host.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp]
+        L.tl3_spmm_static_scratch.argtypes = [vp, vp, i64, vp, i64, ci, vp]
+        L.tl3_static_scratch_status.argtypes = [vp]
         L.tl3_status.argtypes = [vp, vp, vp]
         L.tl3_last_launch.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci)]
         L.tl3_strerror.argtypes = [ci]
@@ -236,6 +239,24 @@ class Matrix:
                 workspace = self._workspaces[key] = self.new_workspace(N, stream)
         _check(lib().tl3_spmm(self._h, X.data_ptr(), X.stride(0), Y.data_ptr(), Y.stride(0), N,
                               workspace.data_ptr(), _stream_ptr(stream)), "tl3_spmm")
+        return Y
+
+    def spmm_static_scratch(self, X, Y=None, stream=None):
+        """``Y = W X`` without a caller-supplied workspace and without any allocation inside the
+        library: the scratch is a fixed 3 MiB array in the library image (see ``tl3.h``).  Raises
+        ``Tl3Error(ERR_SCRATCH_LIMIT)`` when the problem needs more.  Calls must not overlap on the
+        GPU.  (``Y`` is allocated here, by torch, only if the caller passes none.)"""
+        import torch
+        if X.dtype != torch.float16 or X.dim() != 2 or X.stride(1) != 1:
+            raise ValueError("X must be a 2-D float16 tensor with contiguous rows")
+        M, K = self.shape
+        if X.shape[0] != K:
+            raise ValueError("X has the wrong number of rows")
+        N = X.shape[1]
+        if Y is None:
+            Y = torch.empty((M, N), dtype=torch.float16, device=X.device)
+        _check(lib().tl3_spmm_static_scratch(self._h, X.data_ptr(), X.stride(0), Y.data_ptr(), Y.stride(0), N,
+                                             _stream_ptr(stream)), "tl3_spmm_static_scratch")
         return Y
 
     def spmm_host(self, X: np.ndarray, Y: np.ndarray, dX, dY, workspace, stream=None) -> None:
