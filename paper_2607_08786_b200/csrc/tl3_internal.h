@@ -47,9 +47,10 @@ namespace tl3 {
 //                    bits 0-15 = nibbles of windows 8kb+4h .. 8kb+4h+3 of row (L&7)+16(L>>4),
 //                    bits 16-31 = the same windows of that row + 8, with h = (L>>3)&1
 //   +18432  u32[4]: pdd_len, res_cnt, 0, 0
-//   +18448  chain starts u32[128]: tau0 | rho0 << 16 (0xFFFFFFFF = empty chain)
-//   +18960  chain lengths u8[128]
-//   +19088  PDD delta bytes, chain-major, padded to 4 bytes
+//   +18448  chain starts u32[128]: tau0 | rho0 << 16 (0xFFFFFFFF = empty chain), chains sorted
+//           longest first (ties: lower row first)
+//   +18960  chain lengths u8[128], same order
+//   +19088  PDD delta bytes, chain after chain in that order, padded to 4 bytes
 //   +...    Residual entries u32[res_cnt]: rho | value << 16, padded to 16 bytes
 constexpr int kTileM = 128, kTileK = 128, kH = 64;
 constexpr uint32_t kValsBytes = 16384, kMetaOff = 16384, kMetaBytes = 2048;

@@ -1,6 +1,7 @@
 // Device packer: lays the canonical container out as one blob of per-tile blocks, each ready for
 // a single bulk copy into shared memory (layout described in tl3_internal.h).  The blob is a
 // permutation of the canonical bytes plus alignment padding; nothing is re-encoded.
+#include <algorithm>
 #include <cstring>
 
 #include "tl3_internal.h"
@@ -68,12 +69,28 @@ void pack_device_blob(const tl3_matrix* m, uint8_t* out) {
       uint32_t* info = reinterpret_cast<uint32_t*>(blk + kInfoOff);
       info[0] = pdd_len;
       info[1] = res_cnt;
-      uint32_t* hdrs = reinterpret_cast<uint32_t*>(blk + kHdrOff);
-      for (int r = 0; r < kTileM; ++r) {
-        hdrs[r] = static_cast<uint32_t>(m->chain_tau0[t * kTileM + r]) | static_cast<uint32_t>(m->chain_rho0[t * kTileM + r]) << 16;
-        blk[kLenOff + r] = m->chain_len[t * kTileM + r];
+      // Chains are stored longest first (ties: lower row first).  A decode thread takes the chain at
+      // its own index, so the 32 lanes of a warp get chains of similar length and few lanes idle
+      // while the longest one finishes.  Which row a chain belongs to is carried by its rho values.
+      int order[kTileM];
+      uint32_t start[kTileM];
+      {
+        uint32_t acc = 0;
+        for (int r = 0; r < kTileM; ++r) { order[r] = r; start[r] = acc; acc += m->chain_len[t * kTileM + r]; }
+        std::stable_sort(order, order + kTileM, [&](int a, int b) {
+          return m->chain_len[t * kTileM + a] > m->chain_len[t * kTileM + b];
+        });
       }
-      if (pdd_len) std::memcpy(blk + kPddOff, &m->pdd_bytes[pdd_off], pdd_len);
+      uint32_t* hdrs = reinterpret_cast<uint32_t*>(blk + kHdrOff);
+      uint8_t* code = blk + kPddOff;
+      for (int j = 0; j < kTileM; ++j) {
+        const int r = order[j];
+        const uint32_t len = m->chain_len[t * kTileM + r];
+        hdrs[j] = static_cast<uint32_t>(m->chain_tau0[t * kTileM + r]) | static_cast<uint32_t>(m->chain_rho0[t * kTileM + r]) << 16;
+        blk[kLenOff + j] = static_cast<uint8_t>(len);
+        if (len) std::memcpy(code, &m->pdd_bytes[pdd_off + start[r]], len);
+        code += len;
+      }
       uint32_t* res = reinterpret_cast<uint32_t*>(blk + kPddOff + align_up(pdd_len, 4));
       for (uint32_t j = 0; j < res_cnt; ++j)
         res[j] = static_cast<uint32_t>(m->res_rho[res_off + j]) | static_cast<uint32_t>(m->res_val[res_off + j]) << 16;

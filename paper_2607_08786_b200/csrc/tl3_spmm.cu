@@ -7,12 +7,12 @@
 //     with ONE bulk copy and the matching 128 x N block of X with one TMA tensor copy into a ring
 //     of shared-memory stages (Sec. 4.2 "Efficient Matrix Loading": W streamed tile by tile, X
 //     small enough to live in L2);
-//   * two groups of four decode warps alternate over the tiles: copy the 2-bit metadata to tensor
+//   * four groups of four decode warps take the tiles in turn: copy the 2-bit metadata to tensor
 //     memory, run Algorithm 1 (one PDD chain per thread; chain byte offsets by a warp-shuffle
 //     prefix sum of the chain lengths) moving each parked value from W_t to a second 2:4 operand
 //     W_r and zeroing its slot, and scatter the Residual entries into W_r as well
 //     (Sec. 4.3; surplus weights always sit at in-window index 2 or 3, so W_r's metadata is the
-//     constant pattern {2,3});
+//     constant pattern {2,3}); two more warps clear each W_r buffer as soon as its MMAs are done;
 //   * one thread issues tcgen05.mma.sp (kind::f16, M = 128, K = 32) on W_t and on W_r into the
 //     same fp32 accumulator in tensor memory (Sec. 4.3 "Sparse TC Computation");
 //   * four epilogue warps read the accumulator; a row-tile owned by one CTA is written to Y
@@ -25,7 +25,6 @@
 #include <cuda_fp16.h>
 
 #include <cstdint>
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <vector>
@@ -52,15 +51,16 @@ void set_cuda_error(int e) { g_last_cuda_error = e; }
 constexpr int kGroups = 4;                // decode groups of four warps; tile i goes to group i % 4
 constexpr int kProducerWarp = 0;
 constexpr int kMmaWarp = 1;
-constexpr int kAllocWarp = 2;             // warp 3 is idle; decode groups start at a multiple of four warps
-                                          // because a warp reaches tensor-memory lanes 32*(warp%4)..+31
+constexpr int kAllocWarp = 2;
+constexpr int kClearWarp0 = 2;            // warps 2 and 3 clear the W_r buffers (warp 2 also owns the TMEM allocation)
+                                          // decode groups start at a multiple of four warps because a
+                                          // warp reaches tensor-memory lanes 32*(warp%4)..+31
 constexpr int kDecodeWarp0 = 4;           // warps 4-7: decode group 0, 8-11: group 1, ...
 constexpr int kEpilogueWarp0 = kDecodeWarp0 + 4 * kGroups;
 constexpr int kThreads = (kEpilogueWarp0 + 4) * 32;
 constexpr int kMaxStages = 8;
 constexpr uint32_t kWrBytes = 16384;
 constexpr int kWrBuffers = 4;             // W_r ring: tile i uses buffer i % 4
-static_assert(kWrBuffers % kGroups == 0, "a W_r buffer must always belong to the same decode group");
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColMetaT = 128;       // + 4 * (tile % 4): metadata of W_t, four columns per tile in flight
 constexpr uint32_t kColMetaR = 144;       // two columns of 0xEEEEEEEE
@@ -71,7 +71,7 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per kernel
 // status codes written to the workspace status word (0 = ok)
 enum : uint32_t {
   kStProducer = 1, kStDecodeFull = 2, kStDecodeWrFree = 3, kStMmaDecoded = 4, kStMmaAccEmpty = 5,
-  kStEpilogueAccFull = 6, kStDrain = 7
+  kStEpilogueAccFull = 6, kStDrain = 7, kStClearWrFree = 8, kStDecodeWrReady = 9
 };
 
 struct KernelArgs {
@@ -89,7 +89,6 @@ struct KernelArgs {
   uint32_t x_offset;         // offset of the X tile inside a stage, multiple of 1024
   int num_stages;
   long long* timing;         // phase-timing buffer (debug builds), else null
-  int debug_skip;            // debug builds: bit 0 skips the W_t MMAs, bit 1 the W_r MMAs, bit 2 the chain decode
 };
 
 // Optional per-role phase timing (build with -DTL3_PHASE_TIMING): CTA 0 adds the clock cycles it
@@ -99,10 +98,8 @@ static long long* g_timing_buffer = nullptr;
 #define TL3_T0() long long tacc_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long tprev_ = clock64();
 #define TL3_TACC(k) { const long long tn_ = clock64(); tacc_[k] += tn_ - tprev_; tprev_ = tn_; }
 #define TL3_TDUMP(base) { if (a.timing && blockIdx.x == 0) for (int q_ = 0; q_ < 8; ++q_) a.timing[(base) + q_] = tacc_[q_]; }
-#define TL3_SKIP(bit) (a.debug_skip & (bit))
 #define TL3_STAMP(tile, k) { if (a.timing && blockIdx.x == 0 && (tile) >= 18 && (tile) < 26) a.timing[200 + 8 * ((tile) - 18) + (k)] = clock64(); }
 #else
-#define TL3_SKIP(bit) false
 #define TL3_STAMP(tile, k) {}
 #define TL3_T0() {}
 #define TL3_TACC(k) {}
@@ -268,45 +265,56 @@ __device__ __forceinline__ void sts_zero16B(uint32_t addr) {
   asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
 }
 
-// Algorithm 1 for one chain, kBatch delta bytes at a time.  `pos` carries offset_t in its low and
-// offset_r in its high 16 bits, so one add advances both cursors.  Within a batch all positions
-// are formed first, then all W_t loads are issued, then all stores, so that the shared-memory
-// round trips of different entries overlap.
+// Algorithm 1 for one chain, eight delta bytes at a time.  `pos` carries offset_t in its low and
+// offset_r in its high 16 bits, so one add advances both cursors and one shift/xor pair forms both
+// swizzled byte offsets.  Within a batch all positions are formed first, then all W_t loads are
+// issued, then all stores, so that the shared-memory round trips of different entries overlap; the
+// code words of the next batch are fetched before the current one is processed.
 constexpr int kBatch = 8;
+
+// packed byte offsets (W_t offset low, W_r offset high) of the packed positions `pos`
+__device__ __forceinline__ uint32_t swizzled_offset2(uint32_t pos) { return (pos << 1) ^ ((pos >> 2) & 0x00700070u); }
 
 __device__ __forceinline__ void decode_chain(uint32_t stage, uint32_t wr, uint32_t hdr, uint32_t code_addr, uint32_t len) {
   if (hdr == 0xFFFFFFFFu) return;                       // empty chain
   uint32_t pos = hdr;
-  {                                                     // first pair: absolute 16-bit positions
-    const uint32_t at = stage + swizzled_offset(pos & 0xFFFFu);
-    const uint32_t v = lds_u16(at);
-    sts_u16(at, 0);                                     // W_t[offset_t] = 0
-    sts_u16(wr + swizzled_offset(pos >> 16), v);        // W_r[offset_r] = W_t[offset_t]
-  }
   uint32_t word_addr = code_addr & ~3u;
   const uint32_t shift = (code_addr & 3u) * 8u;
+  uint32_t w0 = 0, w1 = 0, w2 = 0;
+  if (len != 0) { w0 = lds_u32(word_addr); w1 = lds_u32(word_addr + 4); w2 = lds_u32(word_addr + 8); }
+  {                                                     // first pair: absolute 16-bit positions
+    const uint32_t off2 = swizzled_offset2(pos);
+    const uint32_t at = stage + (off2 & 0xFFFFu);
+    const uint32_t v = lds_u16(at);
+    sts_u16(at, 0);                                     // W_t[offset_t] = 0
+    sts_u16(wr + (off2 >> 16), v);                      // W_r[offset_r] = W_t[offset_t]
+  }
   for (uint32_t k0 = 0; k0 < len; k0 += kBatch) {
-    const uint32_t w0 = lds_u32(word_addr), w1 = lds_u32(word_addr + 4), w2 = lds_u32(word_addr + 8);
-    word_addr += kBatch;
-    const uint32_t bytes[2] = {__funnelshift_r(w0, w1, shift), __funnelshift_r(w1, w2, shift)};
-    uint32_t at[kBatch], ar[kBatch], val[kBatch];
+    uint32_t lo = __funnelshift_r(w0, w1, shift), hi = __funnelshift_r(w1, w2, shift);
+    const uint32_t rem = len - k0;
+    if (rem > kBatch) {                                 // code words of the next batch
+      word_addr += kBatch;
+      w0 = w2; w1 = lds_u32(word_addr + 4); w2 = lds_u32(word_addr + 8);
+    } else if (rem < kBatch) {                          // bytes past the end behave like dummies
+      if (rem <= 4) { hi = 0; if (rem < 4) lo &= (1u << (8 * rem)) - 1u; }
+      else hi &= (1u << (8 * (rem - 4))) - 1u;
+    }
+    uint32_t off2[kBatch], val[kBatch];
     bool real[kBatch];
 #pragma unroll
     for (int q = 0; q < kBatch; ++q) {
-      uint32_t bt = (bytes[q >> 2] >> (8 * (q & 3))) & 0xFFu;
-      bt = (k0 + q < len) ? bt : 0u;                    // past the end: behaves like a dummy
-      const uint32_t dt = bt & 0xFu, dr = bt >> 4;
-      pos += dt | (dr << 16);
-      real[q] = (dt != 0u) && (dr != 0u);               // a zero nibble marks a dummy point
-      at[q] = stage + swizzled_offset(pos & 0xFFFFu);
-      ar[q] = wr + swizzled_offset(pos >> 16);
+      const uint32_t bt = __byte_perm(q < 4 ? lo : hi, 0u, 0x4440u + (q & 3));   // delta byte q
+      const uint32_t delta = (bt * 0x1001u) & 0x000F000Fu;      // t delta | r delta << 16
+      pos += delta;
+      real[q] = ((delta - 0x00010001u) & 0x80008000u) == 0u;    // both nibbles non-zero (else a dummy point)
+      off2[q] = swizzled_offset2(pos);
     }
 #pragma unroll
     for (int q = 0; q < kBatch; ++q)
-      if (real[q]) val[q] = lds_u16(at[q]);
+      if (real[q]) val[q] = lds_u16(stage + (off2[q] & 0xFFFFu));
 #pragma unroll
     for (int q = 0; q < kBatch; ++q)
-      if (real[q]) { sts_u16(at[q], 0); sts_u16(ar[q], val[q]); }
+      if (real[q]) { sts_u16(stage + (off2[q] & 0xFFFFu), 0); sts_u16(wr + (off2[q] >> 16), val[q]); }
   }
 }
 
@@ -318,10 +326,10 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   const int S = a.num_stages;
   uint8_t* wr_base = smem + static_cast<size_t>(S) * a.stage_stride;           // kWrBuffers x 16 KB
   uint8_t* bar_base = wr_base + kWrBuffers * kWrBytes;
-  // barrier block: full[8] mma_done[8] decoded[8] acc_full[2] acc_empty[2] | tmem slot | flags
+  // barrier block: full[8] mma_done[8] decoded[8] acc_full[2] acc_empty[2] wr_ready[4] | tmem slot | flags
   uint64_t* bars = reinterpret_cast<uint64_t*>(bar_base);
   const uint32_t bar_full = smem_u32(bars), bar_mma = smem_u32(bars + 8), bar_dec = smem_u32(bars + 16);
-  const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26);
+  const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26), bar_wrready = smem_u32(bars + 28);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 32);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 33);
   volatile unsigned int* last_flag = reinterpret_cast<volatile unsigned int*>(bars + 34);
@@ -343,6 +351,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       mbar_init(bar_accfull + 8 * b, 1);
       mbar_init(bar_accempty + 8 * b, 128);
     }
+    for (int w = 0; w < kWrBuffers; ++w) mbar_init(bar_wrready + 8 * w, 64);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -380,9 +389,9 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         const uint32_t full = bar_full + 8 * s;
         const uint8_t* src = a.blob + static_cast<size_t>(off16) * 16;
         if (elect_one()) {
-          mbar_arrive_expect_tx(full, bytes + (TL3_SKIP(64) ? 0u : 128u * NPAD * 2u));
+          mbar_arrive_expect_tx(full, bytes + 128u * NPAD * 2u);
           bulk_copy_g2s(stage, src, bytes, full);
-          if (!TL3_SKIP(64)) tma_load_2d(stage + a.x_offset, &x_map, 0, kt * kTileK, full);
+          tma_load_2d(stage + a.x_offset, &x_map, 0, kt * kTileK, full);
           TL3_STAMP(i, 1)
         }
         __syncwarp();
@@ -403,6 +412,28 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
           if (global_timer() - t1 > kWaitLimitNs / 4) { atomicCAS(a.status, 0u, (uint32_t)kStDrain); break; }
         }
       }
+    }
+  } else if (warp == kClearWarp0 || warp == kClearWarp0 + 1) {
+    // ------------------------------------------------------------------ W_r clearing
+    // Tile i scatters into W_r buffer i % 4.  These two warps zero a buffer as soon as the MMAs
+    // of tile i - 4 (its previous user) are done and then open it for the decode warps, so the
+    // decode path neither clears nor needs a group-wide barrier.
+    const int ct = tid - kClearWarp0 * 32;                       // 0..63
+    const uint32_t wr0 = smem_u32(wr_base);
+    int s4 = 0;                                                  // stage and phase of tile i - kWrBuffers
+    uint32_t ph4 = 0;
+    for (int i = 0; i < n_tiles; ++i) {
+      const int wb = i & (kWrBuffers - 1);
+      bool ok = true;
+      if (i >= kWrBuffers) {
+        ok = mbar_wait(bar_mma + 8 * s4, ph4, wctx, kStClearWrFree);
+        if (++s4 == S) { s4 = 0; ph4 ^= 1u; }
+      }
+      if (!__all_sync(0xFFFFFFFFu, ok)) break;
+      const uint32_t wr = wr0 + wb * kWrBytes;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) sts_zero16B(wr + (c * 64 + ct) * 16);
+      mbar_arrive(bar_wrready + 8 * wb);
     }
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
@@ -444,9 +475,9 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb) {
           const uint32_t id = idesc | static_cast<uint32_t>(kb & 1);
-          if (!TL3_SKIP(1)) umma_sp_f16(d_tmem, a_lo + kb * kAStep, kAHi, b_lo + kb * kBStep, kBHi, e_t + (kb & ~1), id,
-                                        (first_of_seg && kb == 0) ? 0u : 1u);
-          if (!TL3_SKIP(2)) umma_sp_f16(d_tmem, w_lo + kb * kAStep, kAHi, b_lo + kb * kBStep, kBHi, e_r, id, 1u);
+          umma_sp_f16(d_tmem, a_lo + kb * kAStep, kAHi, b_lo + kb * kBStep, kBHi, e_t + (kb & ~1), id,
+                      (first_of_seg && kb == 0) ? 0u : 1u);
+          umma_sp_f16(d_tmem, w_lo + kb * kAStep, kAHi, b_lo + kb * kBStep, kBHi, e_r, id, 1u);
         }
         umma_commit(mma_bar);         // frees the stage, this tile's W_r buffer and metadata columns
         if (last_of_seg) umma_commit(acc_bar);
@@ -470,35 +501,35 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};"
                    ::"r"(tmem_base + lane_base + kColMetaR), "r"(0xEEEEEEEEu), "r"(0xEEEEEEEEu) : "memory");
     }
-    constexpr int kHist = kWrBuffers / kGroups;                  // own tiles between two uses of a W_r buffer
-    int s = g % S, hist_s[kHist];
-    uint32_t ph = (g / S) & 1, hist_ph[kHist];
-#pragma unroll
-    for (int h = 0; h < kHist; ++h) { hist_s[h] = 0; hist_ph[h] = 0; }
+    static_assert(kWrBuffers == kGroups, "tile i of group i % kGroups uses W_r buffer i % kWrBuffers");
+    const int wb = g;                                           // this group's W_r buffer and metadata columns
+    const uint32_t wr = wr0 + wb * kWrBytes;
+    int s = g % S;
+    uint32_t ph = (g / S) & 1;
     TL3_T0()
-    for (int i = g; i < n_tiles; i += kGroups) {
+    for (int i = g, j = 0; i < n_tiles; i += kGroups, ++j) {
       TL3_TACC(0)
-      const int wb = i & (kWrBuffers - 1);
-      const uint32_t wr = wr0 + wb * kWrBytes;
-      // this W_r buffer and its metadata columns were last read by the MMAs of tile i - 4
-      bool ok = (i < kWrBuffers) || mbar_wait(bar_mma + 8 * hist_s[kHist - 1], hist_ph[kHist - 1], wctx, kStDecodeWrFree);
+      // Warps of a group do not wait for each other.  The packed block lists chains longest
+      // first, so the four warps get blocks of different length; the block a warp takes rotates
+      // from tile to tile to even the load out.
+      const int cr = (r + 32 * (j & 3)) & 127;                  // chain handled by this thread
+      bool ok = mbar_wait(bar_full + 8 * s, ph, wctx, kStDecodeFull);
       TL3_TACC(1)
-      if (ok && !TL3_SKIP(8)) {   // clear W_r, 16 bytes per thread and step, consecutive threads -> consecutive chunks
-#pragma unroll
-        for (int c = 0; c < 8; ++c) sts_zero16B(wr + (c * 128 + r) * 16);
-      }
-      TL3_TACC(2)
-      ok = ok && mbar_wait(bar_full + 8 * s, ph, wctx, kStDecodeFull);
-      TL3_TACC(3)
-      // W_r must be clear before anyone scatters into it; the same barrier makes the give-up
-      // decision uniform across the group.
-      if (!named_bar_all(1 + g, 128, ok)) break;
-      if (r == 0) TL3_STAMP(i, 2)
       const uint32_t stage = smem_base + static_cast<uint32_t>(s) * a.stage_stride;
-      // metadata -> tensor memory (4 columns of this group)
-      if (!TL3_SKIP(16)) {
-        uint32_t m0, m1, m2, m3;
+      uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0, quad = 0, hdr = 0xFFFFFFFFu;
+      if (ok) {
         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(m0), "=r"(m1), "=r"(m2), "=r"(m3) : "r"(stage + kMetaOff + r * 16));
+        quad = lds_u32(stage + kLenOff + lane * 4);
+        hdr = lds_u32(stage + kHdrOff + cr * 4);
+      }
+      // the W_r buffer was cleared after the MMAs of tile i - 4 finished; the same event freed
+      // the metadata columns
+      ok = ok && mbar_wait(bar_wrready + 8 * wb, j & 1, wctx, kStDecodeWrReady);
+      TL3_TACC(2)
+      if (!__all_sync(0xFFFFFFFFu, ok)) break;
+      if (r == 0) TL3_STAMP(i, 2)
+      // metadata -> tensor memory (4 columns of this group)
+      {
         asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
                      ::"r"(tmem_base + lane_base + kColMetaT + 4 * wb), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
       }
@@ -506,7 +537,6 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       // Each warp scans all 128 lengths (4 per lane) with shuffles; no cross-warp exchange.
       uint32_t off, len;
       {
-        const uint32_t quad = lds_u32(stage + kLenOff + lane * 4);
         const uint32_t qsum = __dp4a(quad, 0x01010101u, 0u);
         uint32_t incl = qsum;
 #pragma unroll
@@ -514,19 +544,19 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
           const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl, d);
           if (lane >= d) incl += n;
         }
-        const int src = r >> 2;                                  // lane that holds my quad
+        const int src = cr >> 2;                                 // lane that holds my chain's quad
         const uint32_t q = __shfl_sync(0xFFFFFFFFu, quad, src);
         const uint32_t excl = __shfl_sync(0xFFFFFFFFu, incl - qsum, src);
-        const int sub = r & 3;
+        const int sub = cr & 3;
         off = excl + __dp4a(q & ((1u << (8 * sub)) - 1u), 0x01010101u, 0u);
         len = (q >> (8 * sub)) & 0xFFu;
       }
       TL3_TACC(4)
-      if (!TL3_SKIP(4)) decode_chain(stage, wr, lds_u32(stage + kHdrOff + r * 4), stage + kPddOff + off, len);
+      decode_chain(stage, wr, hdr, stage + kPddOff + off, len);
       __syncwarp();
       TL3_TACC(5)
       // Residual layer: (position, value) entries go to W_r too
-      if (!TL3_SKIP(32)) {
+      {
         const uint32_t pdd_len = lds_u32(stage + kInfoOff), res_cnt = lds_u32(stage + kInfoOff + 4);
         const uint32_t res = stage + kPddOff + ((pdd_len + 3u) & ~3u);
         for (uint32_t k = r; k < res_cnt; k += 128) {
@@ -541,9 +571,6 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       mbar_arrive(bar_dec + 8 * s);
       if (r == 0) TL3_STAMP(i, 3)
       TL3_TACC(7)
-#pragma unroll
-      for (int h = kHist - 1; h > 0; --h) { hist_s[h] = hist_s[h - 1]; hist_ph[h] = hist_ph[h - 1]; }
-      hist_s[0] = s; hist_ph[0] = ph;
       s += kGroups;
       while (s >= S) { s -= S; ph ^= 1u; }
     }
@@ -828,10 +855,8 @@ int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t l
   args.num_stages = stages;
 #ifdef TL3_PHASE_TIMING
   args.timing = g_timing_buffer;
-  args.debug_skip = getenv("TL3_DEBUG_SKIP") ? atoi(getenv("TL3_DEBUG_SKIP")) : 0;
 #else
   args.timing = nullptr;
-  args.debug_skip = 0;
 #endif
   m->last_ctas = grid; m->last_stages = stages; m->last_smem = static_cast<int>(smem_bytes);
   cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -169,7 +169,12 @@ def _expected_blob_blocks(c, M_pad, K_pad):
             hdr = (c.chain_tau0[t * 128:(t + 1) * 128].astype(np.uint32) |
                    c.chain_rho0[t * 128:(t + 1) * 128].astype(np.uint32) << 16)
             lens = c.chain_len[t * 128:(t + 1) * 128]
-            pdd = c.pdd_bytes[pdd_off:pdd_off + pdd_len]
+            # chains longest first, ties by row
+            order = sorted(range(128), key=lambda r: (-int(lens[r]), r))
+            starts = np.concatenate([[0], np.cumsum(lens.astype(np.int64))])
+            codes = c.pdd_bytes[pdd_off:pdd_off + pdd_len]
+            pdd = np.concatenate([codes[starts[r]:starts[r + 1]] for r in order]) if pdd_len else codes
+            hdr, lens = hdr[order], lens[order]
             pad = (-pdd_len) % 4
             res = (c.res_rho[res_off:res_off + res_cnt].astype(np.uint32) |
                    c.res_val[res_off:res_off + res_cnt].astype(np.uint32) << 16)
