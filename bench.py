@@ -221,6 +221,9 @@ def run_ours(args, rank, local_rank, world):
     dist.barrier()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop()
+    for L in launches:
+        word = L["m"].status_word(L["ws"])
+        assert word == 0, f"kernel status word {word:#x} for {L['case'].name}"
     ms_total = dist.max_over_ranks(ms_total, device=dev)
     ms_step = ms_total / args.steps
     step_bytes = sum(L["bytes"] for L in launches)

@@ -163,9 +163,13 @@ int tl3_spmm_static_scratch(const tl3_matrix* m, const void* X, int64_t ldx, voi
                             void* stream);
 int tl3_static_scratch_status(void* stream);
 
-/* Read the workspace's status word (synchronises `stream`).  TL3_OK, or DEVICE_TIMEOUT if a
- * bounded wait inside a kernel expired since the last tl3_workspace_init(). */
+/* Read the workspace's status word (synchronises `stream`).  TL3_OK; DEVICE_TIMEOUT if a bounded
+ * wait inside a kernel expired since the last tl3_workspace_init(); BAD_CONTAINER if the decoder
+ * met a block whose lengths or decoded positions were out of range (it skips such entries rather
+ * than touching memory outside the tile).  tl3_status_word() also hands back the raw word:
+ * bits 0-7 = code (1-9: which wait gave up, 16: bad block), higher bits = detail. */
 int tl3_status(const tl3_matrix* m, void* workspace, void* stream);
+int tl3_status_word(void* workspace, void* stream, uint32_t* word);
 
 /* Kernel launch geometry of the last tl3_spmm on this handle (for reporting): CTAs, stages. */
 int tl3_last_launch(const tl3_matrix* m, int* ctas, int* stages, int* smem_bytes);

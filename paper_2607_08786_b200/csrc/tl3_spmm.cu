@@ -71,7 +71,8 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per kernel
 // status codes written to the workspace status word (0 = ok)
 enum : uint32_t {
   kStProducer = 1, kStDecodeFull = 2, kStDecodeWrFree = 3, kStMmaDecoded = 4, kStMmaAccEmpty = 5,
-  kStEpilogueAccFull = 6, kStDrain = 7, kStClearWrFree = 8, kStDecodeWrReady = 9
+  kStEpilogueAccFull = 6, kStDrain = 7, kStClearWrFree = 8, kStDecodeWrReady = 9,
+  kStBadBlock = 16           // a block's lengths or a decoded position were out of range (+ detail in bits 8..)
 };
 
 struct KernelArgs {
@@ -275,8 +276,11 @@ constexpr int kBatch = 8;
 // packed byte offsets (W_t offset low, W_r offset high) of the packed positions `pos`
 __device__ __forceinline__ uint32_t swizzled_offset2(uint32_t pos) { return (pos << 1) ^ ((pos >> 2) & 0x00700070u); }
 
-__device__ __forceinline__ void decode_chain(uint32_t stage, uint32_t wr, uint32_t hdr, uint32_t code_addr, uint32_t len) {
+// Positions are checked (< 8192 slots per tile) before they become addresses; a violation is
+// reported in *bad and the entry is skipped.
+__device__ __forceinline__ void decode_chain(uint32_t stage, uint32_t wr, uint32_t hdr, uint32_t code_addr, uint32_t len, uint32_t* bad) {
   if (hdr == 0xFFFFFFFFu) return;                       // empty chain
+  if (hdr & 0xE000E000u) { *bad = 1u; return; }
   uint32_t pos = hdr;
   uint32_t word_addr = code_addr & ~3u;
   const uint32_t shift = (code_addr & 3u) * 8u;
@@ -307,6 +311,7 @@ __device__ __forceinline__ void decode_chain(uint32_t stage, uint32_t wr, uint32
       const uint32_t delta = (bt * 0x1001u) & 0x000F000Fu;      // t delta | r delta << 16
       pos += delta;
       real[q] = ((delta - 0x00010001u) & 0x80008000u) == 0u;    // both nibbles non-zero (else a dummy point)
+      if (pos & 0xE000E000u) { real[q] = false; *bad = 2u; }
       off2[q] = swizzled_offset2(pos);
     }
 #pragma unroll
@@ -326,10 +331,10 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   const int S = a.num_stages;
   uint8_t* wr_base = smem + static_cast<size_t>(S) * a.stage_stride;           // kWrBuffers x 16 KB
   uint8_t* bar_base = wr_base + kWrBuffers * kWrBytes;
-  // barrier block: full[8] mma_done[8] decoded[8] acc_full[2] acc_empty[2] wr_ready[4] | tmem slot | flags
+  // barrier block: full[8] mma_done[8] decoded[8] acc_full[2] acc_empty[2] wr_ready[4] | tmem slot | flags | wr_free[4]
   uint64_t* bars = reinterpret_cast<uint64_t*>(bar_base);
   const uint32_t bar_full = smem_u32(bars), bar_mma = smem_u32(bars + 8), bar_dec = smem_u32(bars + 16);
-  const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26), bar_wrready = smem_u32(bars + 28);
+  const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26), bar_wrready = smem_u32(bars + 28), bar_wrfree = smem_u32(bars + 36);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 32);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 33);
   volatile unsigned int* last_flag = reinterpret_cast<volatile unsigned int*>(bars + 34);
@@ -339,6 +344,10 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   const long long t_begin = range_begin(blockIdx.x, T, G), t_end = range_begin(blockIdx.x + 1, T, G);
   const int n_tiles = static_cast<int>(t_end - t_begin);
   const int kt_begin = static_cast<int>(t_begin % a.tiles_k);
+  // Decode groups in use: a group may wait for its next tile only once the stage's previous
+  // phase has completed (a parity wait cannot tell phases two apart), which holds as long as
+  // there are no more groups than stages.  Tile i goes to group i % AG and W_r buffer i % AG.
+  const int AG = S < kGroups ? S : kGroups;
   const uint32_t smem_base = smem_u32(smem);
 
   if (tid == 0) {
@@ -351,7 +360,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       mbar_init(bar_accfull + 8 * b, 1);
       mbar_init(bar_accempty + 8 * b, 128);
     }
-    for (int w = 0; w < kWrBuffers; ++w) mbar_init(bar_wrready + 8 * w, 64);
+    for (int w = 0; w < kWrBuffers; ++w) { mbar_init(bar_wrready + 8 * w, 64); mbar_init(bar_wrfree + 8 * w, 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -415,25 +424,23 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     }
   } else if (warp == kClearWarp0 || warp == kClearWarp0 + 1) {
     // ------------------------------------------------------------------ W_r clearing
-    // Tile i scatters into W_r buffer i % 4.  These two warps zero a buffer as soon as the MMAs
-    // of tile i - 4 (its previous user) are done and then open it for the decode warps, so the
-    // decode path neither clears nor needs a group-wide barrier.
+    // Tile i scatters into W_r buffer i % AG.  These two warps zero a buffer as soon as the MMAs
+    // of tile i - AG (its previous user) are done (the MMA warp commits to the buffer's own
+    // barrier) and then open it for the decode warps, so the decode path neither clears nor needs
+    // a group-wide barrier.
     const int ct = tid - kClearWarp0 * 32;                       // 0..63
     const uint32_t wr0 = smem_u32(wr_base);
-    int s4 = 0;                                                  // stage and phase of tile i - kWrBuffers
-    uint32_t ph4 = 0;
+    int wb = 0, use = 0;                                         // buffer of tile i, and how often it was filled before
     for (int i = 0; i < n_tiles; ++i) {
-      const int wb = i & (kWrBuffers - 1);
       bool ok = true;
-      if (i >= kWrBuffers) {
-        ok = mbar_wait(bar_mma + 8 * s4, ph4, wctx, kStClearWrFree);
-        if (++s4 == S) { s4 = 0; ph4 ^= 1u; }
-      }
+      if (use >= 1) ok = mbar_wait(bar_wrfree + 8 * wb, (use - 1) & 1, wctx, kStClearWrFree);
       if (!__all_sync(0xFFFFFFFFu, ok)) break;
       const uint32_t wr = wr0 + wb * kWrBytes;
 #pragma unroll
       for (int c = 0; c < 16; ++c) sts_zero16B(wr + (c * 64 + ct) * 16);
+      fence_proxy_async_smem();                                  // the MMA reads what stays zero
       mbar_arrive(bar_wrready + 8 * wb);
+      if (++wb == AG) { wb = 0; ++use; }
     }
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
@@ -452,13 +459,13 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     constexpr uint32_t kAStep = 32u >> 4, kBStep = (32u * NPAD * 2u) >> 4;
     const uint32_t a_lo0 = (smem_base >> 4) | kLboOne, stride16 = a.stage_stride >> 4, x16 = a.x_offset >> 4;
     const uint32_t w_lo0 = (smem_u32(wr_base) >> 4) | kLboOne;
-    int seg = 0, s = 0, kt = kt_begin;
+    int seg = 0, s = 0, kt = kt_begin, wb = 0;
     uint32_t ph = 0, a_lo = a_lo0;
     TL3_T0()
     for (int i = 0; i < n_tiles; ++i) {
       const bool first_of_seg = (i == 0) || (kt == 0);
       const bool last_of_seg = (i == n_tiles - 1) || (kt == a.tiles_k - 1);
-      const int b = seg & 1, wb = i & (kWrBuffers - 1);
+      const int b = seg & 1;
       bool ok = true;
       if (first_of_seg && (seg >> 1) >= 1) ok = mbar_wait(bar_accempty + 8 * b, ((seg >> 1) - 1) & 1, wctx, kStMmaAccEmpty);
       TL3_TACC(0)
@@ -470,7 +477,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(b * NPAD);
       const uint32_t e_t = tmem_base + kColMetaT + 4 * wb, e_r = tmem_base + kColMetaR;
       const uint32_t b_lo = a_lo + x16, w_lo = w_lo0 + wb * (kWrBytes >> 4);
-      const uint32_t mma_bar = bar_mma + 8 * s, acc_bar = bar_accfull + 8 * b;
+      const uint32_t mma_bar = bar_mma + 8 * s, acc_bar = bar_accfull + 8 * b, wrfree_bar = bar_wrfree + 8 * wb;
       if (elect_one()) {
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb) {
@@ -479,7 +486,8 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
                       (first_of_seg && kb == 0) ? 0u : 1u);
           umma_sp_f16(d_tmem, w_lo + kb * kAStep, kAHi, b_lo + kb * kBStep, kBHi, e_r, id, 1u);
         }
-        umma_commit(mma_bar);         // frees the stage, this tile's W_r buffer and metadata columns
+        umma_commit(mma_bar);         // frees the stage
+        umma_commit(wrfree_bar);      // frees this tile's W_r buffer and metadata columns
         if (last_of_seg) umma_commit(acc_bar);
       }
       __syncwarp();
@@ -489,6 +497,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       a_lo += stride16;
       if (++s == S) { s = 0; ph ^= 1u; a_lo = a_lo0; }
       if (++kt == a.tiles_k) kt = 0;
+      if (++wb == AG) wb = 0;
     }
     if (lane == 0) TL3_TDUMP(8)
   } else if (warp >= kDecodeWarp0 && warp < kEpilogueWarp0) {
@@ -501,20 +510,27 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};"
                    ::"r"(tmem_base + lane_base + kColMetaR), "r"(0xEEEEEEEEu), "r"(0xEEEEEEEEu) : "memory");
     }
-    static_assert(kWrBuffers == kGroups, "tile i of group i % kGroups uses W_r buffer i % kWrBuffers");
+    static_assert(kWrBuffers == kGroups, "group g owns W_r buffer g");
     const int wb = g;                                           // this group's W_r buffer and metadata columns
     const uint32_t wr = wr0 + wb * kWrBytes;
-    int s = g % S;
-    uint32_t ph = (g / S) & 1;
+    int s = g;                                                  // g < AG <= S
+    uint32_t ph = 0;
     TL3_T0()
-    for (int i = g, j = 0; i < n_tiles; i += kGroups, ++j) {
+    for (int i = g, j = 0; g < AG && i < n_tiles; i += AG, ++j) {
       TL3_TACC(0)
       // Warps of a group do not wait for each other.  The packed block lists chains longest
       // first, so the four warps get blocks of different length; the block a warp takes rotates
       // from tile to tile to even the load out.
       const int cr = (r + 32 * (j & 3)) & 127;                  // chain handled by this thread
-      bool ok = mbar_wait(bar_full + 8 * s, ph, wctx, kStDecodeFull);
+      // Order matters.  The W_r buffer is ready once the MMAs of tile i - AG are done, and MMAs
+      // are issued in tile order, so by then every tile up to i - AG -- in particular the previous
+      // user of this stage, tile i - S -- has been loaded and consumed.  Only then is the parity
+      // wait on the stage's `full` barrier unambiguous (loads may complete out of order, and a
+      // parity wait cannot tell "two phases back" from "done").
+      bool ok = mbar_wait(bar_wrready + 8 * wb, j & 1, wctx, kStDecodeWrReady);
       TL3_TACC(1)
+      ok = ok && mbar_wait(bar_full + 8 * s, ph, wctx, kStDecodeFull);
+      TL3_TACC(2)
       const uint32_t stage = smem_base + static_cast<uint32_t>(s) * a.stage_stride;
       uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0, quad = 0, hdr = 0xFFFFFFFFu;
       if (ok) {
@@ -522,10 +538,6 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         quad = lds_u32(stage + kLenOff + lane * 4);
         hdr = lds_u32(stage + kHdrOff + cr * 4);
       }
-      // the W_r buffer was cleared after the MMAs of tile i - 4 finished; the same event freed
-      // the metadata columns
-      ok = ok && mbar_wait(bar_wrready + 8 * wb, j & 1, wctx, kStDecodeWrReady);
-      TL3_TACC(2)
       if (!__all_sync(0xFFFFFFFFu, ok)) break;
       if (r == 0) TL3_STAMP(i, 2)
       // metadata -> tensor memory (4 columns of this group)
@@ -552,18 +564,24 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         len = (q >> (8 * sub)) & 0xFFu;
       }
       TL3_TACC(4)
-      decode_chain(stage, wr, hdr, stage + kPddOff + off, len);
+      uint32_t bad = 0;
+      const uint32_t pdd_len = lds_u32(stage + kInfoOff), res_cnt = lds_u32(stage + kInfoOff + 4);
+      const uint32_t room = a.x_offset - kPddOff;               // bytes a block may use after its fixed part
+      const bool lens_ok = pdd_len <= room && res_cnt <= room / 4 && ((pdd_len + 3u) & ~3u) + 4u * res_cnt <= room && off + len <= pdd_len;
+      if (lens_ok) decode_chain(stage, wr, hdr, stage + kPddOff + off, len, &bad);
+      else bad = 3u;
       __syncwarp();
       TL3_TACC(5)
       // Residual layer: (position, value) entries go to W_r too
-      {
-        const uint32_t pdd_len = lds_u32(stage + kInfoOff), res_cnt = lds_u32(stage + kInfoOff + 4);
+      if (lens_ok) {
         const uint32_t res = stage + kPddOff + ((pdd_len + 3u) & ~3u);
         for (uint32_t k = r; k < res_cnt; k += 128) {
           const uint32_t rv = lds_u32(res + 4 * k);
-          sts_u16(wr + swizzled_offset(rv & 0xFFFFu), rv >> 16);
+          if ((rv & 0xFFFFu) < 8192u) sts_u16(wr + swizzled_offset(rv & 0xFFFFu), rv >> 16);
+          else bad = 4u;
         }
       }
+      if (bad) atomicCAS(a.status, 0u, kStBadBlock | (bad << 8) | (static_cast<uint32_t>(i) << 12));
       TL3_TACC(6)
       fence_proxy_async_smem();                                   // generic-proxy writes -> MMA reads
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -571,7 +589,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       mbar_arrive(bar_dec + 8 * s);
       if (r == 0) TL3_STAMP(i, 3)
       TL3_TACC(7)
-      s += kGroups;
+      s += AG;
       while (s >= S) { s -= S; ph ^= 1u; }
     }
     if (lane == 0) TL3_TDUMP(16 + 8 * (warp - kDecodeWarp0))
@@ -927,13 +945,21 @@ int tl3_static_scratch_status(void* stream) {
   return tl3_status(nullptr, scratch, stream);
 }
 
-int tl3_status(const tl3_matrix* m, void* workspace, void* stream) {
-  (void)m;
-  if (!workspace) return TL3_ERR_INVALID_ARG;
+int tl3_status_word(void* workspace, void* stream, uint32_t* word) {
+  if (!workspace || !word) return TL3_ERR_INVALID_ARG;
   unsigned int st = 0;
   TL3_CUDA(cudaMemcpyAsync(&st, workspace, sizeof(st), cudaMemcpyDeviceToHost, static_cast<cudaStream_t>(stream)));
   TL3_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
-  return st == 0 ? TL3_OK : TL3_ERR_DEVICE_TIMEOUT;
+  *word = st;
+  return TL3_OK;
+}
+
+int tl3_status(const tl3_matrix* m, void* workspace, void* stream) {
+  (void)m;
+  uint32_t st = 0;
+  if (int rc = tl3_status_word(workspace, stream, &st)) return rc;
+  if (st == 0) return TL3_OK;
+  return (st & 0xFFu) >= tl3::kStBadBlock ? TL3_ERR_BAD_CONTAINER : TL3_ERR_DEVICE_TIMEOUT;
 }
 
 int tl3_last_launch(const tl3_matrix* m, int* ctas, int* stages, int* smem_bytes) {

@@ -136,6 +136,58 @@ def test_degenerate_matrices(tl3, oracle_mod):
     check(oracle_mod, T, X, Y)
 
 
+def test_fewer_stages_than_decode_groups(tl3, oracle_mod):
+    """Large blocks (heavy Residual layer) and a wide X leave room for only two or three stages in
+    shared memory; several tiles per CTA, so the ring wraps many times."""
+    case = wl.Case(0, "s3", 4096, 2048, 64, 3, 0.4, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    Y, m = run_gpu(tl3, W, X, repeats=2)
+    assert m.last_launch()["stages"] <= 3
+    check(oracle_mod, W, X, Y)
+    rng = np.random.default_rng(8)
+    D = (rng.standard_normal((2048, 2048)) * 0.05).astype(np.float16)      # fully dense: half of nnz is Residual
+    D[D == 0] = np.float16(0.01)
+    X = rng.standard_normal((2048, 32)).astype(np.float16)
+    Y, m = run_gpu(tl3, D, X, repeats=2)
+    assert m.last_launch()["stages"] == 2
+    check(oracle_mod, D, X, Y)
+
+
+def test_thousands_of_back_to_back_launches(tl3):
+    """Five different launches in one CUDA graph, replayed without host synchronisation: every
+    replay must leave the status words clear and reproduce the first result bit for bit (the
+    pipeline's barrier protocol must not depend on how loads happen to be ordered in time)."""
+    import torch
+    cases = [wl.Case(0, "a", 2560, 5120, 16, 1, 0.5, "magnitude"), wl.Case(0, "b", 2048, 8192, 32, 2, 0.5, "magnitude"),
+             wl.Case(0, "c", 2048, 2048, 64, 3, 0.4, "magnitude"), wl.Case(0, "d", 1024, 1024, 8, 4, 0.5, "bernoulli"),
+             wl.Case(0, "e", 3000, 3000, 24, 5, 0.7, "magnitude")]
+    L = []
+    for c in cases:
+        m = tl3.encode(c.make_W())
+        m.upload()
+        Xd = device_X(c.make_X())
+        ws = m.new_workspace(c.N)
+        Y = torch.empty((c.M, c.N), dtype=torch.float16, device="cuda")
+        m.spmm(Xd, Y, workspace=ws)
+        torch.cuda.synchronize()
+        L.append((c, m, Xd, Y, ws, Y.clone()))
+
+    def step():
+        for c, m, Xd, Y, ws, ref in L:
+            m.spmm(Xd, Y, workspace=ws)
+
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    for _ in range(5):
+        for _ in range(100):
+            g.replay()
+        torch.cuda.synchronize()
+        for c, m, Xd, Y, ws, ref in L:
+            assert m.status_word(ws) == 0, c.name
+            assert torch.equal(Y, ref), c.name
+
+
 def test_identity_X_reproduces_W_bit_for_bit(tl3):
     """Each y_ij is one product w_ij * 1: the GPU must hand back the decoded W exactly."""
     for k0 in (0, 64):
