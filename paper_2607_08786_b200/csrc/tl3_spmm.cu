@@ -192,6 +192,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
                ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
 
+// Programmatic dependent launch: the next kernel on the stream may be scheduled as soon as every
+// CTA of this one has said so (it still cannot take an SM before a CTA here exits), and a kernel
+// must call pdl_wait() before it reads what its predecessor wrote or writes what its
+// predecessor may still read.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // One lane of a converged warp; the caller keeps every operand warp-uniform so that the
 // single-thread instructions (bulk copies, MMAs, commits) take uniform registers directly.
 __device__ __forceinline__ bool elect_one() {
@@ -373,20 +380,37 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const WaitCtx wctx{abort_flag, a.status, global_timer()};
+  pdl_launch_dependents();
 
   if (warp == kProducerWarp) {
     // ------------------------------------------------------------------ producer
     // The whole warp runs the loop with warp-uniform state; one elected lane issues the copies.
     // Directory entries are read 32 at a time (one per lane) and broadcast with shuffles.
+    // The weight blocks never depend on the kernel that ran before this one, X may: the blocks of
+    // the first S tiles are requested at once, then the warp waits for the predecessor, then X.
     int issued = 0, s = 0, kt = kt_begin;
     uint32_t ph = 0;                                            // phase of the stage's current use
     uint32_t stage = smem_base;
     bool alive = true;
+    const int pre = n_tiles < S ? n_tiles : S;                  // tiles whose stages are free at the start
     TL3_T0()
     for (int base = 0; base < n_tiles && alive; base += 32) {
       uint4 mine = make_uint4(0, 0, 0, 0);
       if (base + lane < n_tiles) mine = __ldg(reinterpret_cast<const uint4*>(a.dir + t_begin + base + lane));
       const int cnt = n_tiles - base < 32 ? n_tiles - base : 32;
+      if (base == 0) {
+        for (int j = 0; j < pre; ++j) {                          // S <= 8 < 32: all in this batch
+          const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.x, j), bytes = __shfl_sync(0xFFFFFFFFu, mine.y, j);
+          const uint8_t* src = a.blob + static_cast<size_t>(off16) * 16;
+          const uint32_t st = smem_base + static_cast<uint32_t>(j) * a.stage_stride, full = bar_full + 8 * j;
+          if (elect_one()) {
+            mbar_arrive_expect_tx(full, bytes + 128u * NPAD * 2u);
+            bulk_copy_g2s(st, src, bytes, full);
+          }
+          __syncwarp();
+        }
+        pdl_wait();
+      }
       for (int j = 0; j < cnt; ++j) {
         const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.x, j), bytes = __shfl_sync(0xFFFFFFFFu, mine.y, j);
         const int i = base + j;
@@ -398,8 +422,10 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         const uint32_t full = bar_full + 8 * s;
         const uint8_t* src = a.blob + static_cast<size_t>(off16) * 16;
         if (elect_one()) {
-          mbar_arrive_expect_tx(full, bytes + 128u * NPAD * 2u);
-          bulk_copy_g2s(stage, src, bytes, full);
+          if (i >= pre) {
+            mbar_arrive_expect_tx(full, bytes + 128u * NPAD * 2u);
+            bulk_copy_g2s(stage, src, bytes, full);
+          }
           tma_load_2d(stage + a.x_offset, &x_map, 0, kt * kTileK, full);
           TL3_STAMP(i, 1)
         }
@@ -599,6 +625,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     int seg = 0;
     long long t = t_begin;
+    pdl_wait();   // Y, the partial sums and the counters may still be in use by the previous kernel
     TL3_T0()
     while (t < t_end) {
       TL3_TACC(0)
@@ -762,7 +789,17 @@ static int launch(const CUtensorMap& map, const KernelArgs& args, int grid, uint
     TL3_CUDA(cudaFuncSetAttribute(tl3_spmm_kernel<NPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemLimit)));
     configured = true;
   }
-  tl3_spmm_kernel<NPAD><<<grid, kThreads, smem_bytes, stream>>>(map, args);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see pdl_wait() in the kernel
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  TL3_CUDA(cudaLaunchKernelEx(&cfg, tl3_spmm_kernel<NPAD>, map, args));
   TL3_CUDA(cudaGetLastError());
   return TL3_OK;
 }
