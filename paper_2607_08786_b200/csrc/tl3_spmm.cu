@@ -67,6 +67,10 @@ constexpr uint32_t kColMetaR = 144;       // two columns of 0xEEEEEEEE
 constexpr uint32_t kSmemLimit = 232448;   // 227 KB
 constexpr uint32_t kBarrierBytes = 1024;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per kernel
+#ifndef TL3_TRYWAIT_HINT_NS
+#define TL3_TRYWAIT_HINT_NS 20000u
+#endif
+constexpr uint32_t kTryWaitHintNs = TL3_TRYWAIT_HINT_NS;     // how long one barrier probe may park the thread
 
 // status codes written to the workspace status word (0 = ok)
 enum : uint32_t {
@@ -136,7 +140,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       "{\n\t.reg .pred q;\n\t"
       "mbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, q;\n\t}"
-      : "=r"(done) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
+      : "=r"(done) : "r"(bar), "r"(parity), "r"(kTryWaitHintNs) : "memory");
   return done != 0;
 }
 
