@@ -386,6 +386,25 @@ def run_ours(args, rank, local_rank, world):
     print(json.dumps(out), flush=True)
 
 
+def run_single(args):
+    """A few launches of one SpMM (for profilers): `--single M K N [--launches L] [--sparsity S]`."""
+    import torch
+    from paper_2607_08786_b200 import build, tl3
+    build.build_library()
+    M, K, N = args.single
+    case = wl.Case(0, f"single_{M}x{K}_n{N}", M, K, N, 6, args.sparsity, "magnitude")
+    m = tl3.encode(case.make_W())
+    m.upload()
+    Xd = torch.from_numpy(case.make_X()).cuda()
+    ws = m.new_workspace(N)
+    Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+    for _ in range(args.launches):
+        m.spmm(Xd, Y, workspace=ws)
+    torch.cuda.synchronize()
+    print(json.dumps({"single": case.name, "launches": args.launches, "status": m.status(ws), **m.last_launch(),
+                      "device_bytes": m.device_bytes()}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -393,7 +412,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--single", type=int, nargs=3, metavar=("M", "K", "N"), help="run a few launches of one shape and exit")
+    ap.add_argument("--launches", type=int, default=3)
+    ap.add_argument("--sparsity", type=float, default=0.5)
     args = ap.parse_args()
+    if args.single:
+        run_single(args)
+        return
     rank, local_rank, world = dist.env_world()
     if args.impl == "reference":
         run_reference(args, rank)
