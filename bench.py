@@ -405,6 +405,112 @@ def run_single(args):
                       "device_bytes": m.device_bytes()}), flush=True)
 
 
+def _time_graph(fn, reps=20):
+    """Device time of fn() per call, as a CUDA graph replayed `reps` times (best of 3)."""
+    import torch
+    fn()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        fn()
+    for _ in range(2):
+        g.replay()
+    torch.cuda.synchronize()
+    best = float("inf")
+    for _ in range(3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1) / reps)
+    return best * 1e3            # microseconds
+
+
+def run_sweep(args):
+    """Extra measurements beside the headline: `--sweep n|sparsity|stack`.  One JSON line per point.
+    Every matrix is uploaded in enough copies that a copy is evicted from L2 before it is used again."""
+    import torch
+    from paper_2607_08786_b200 import build, tl3
+    build.build_library()
+    peak, _ = measured_peak_gbs()
+
+    def point(case, label):
+        W = case.make_W()
+        m0 = tl3.encode(W)
+        copies = max(2, int(np.ceil(3 * 126e6 / m0.device_bytes())))
+        copies = min(copies, 12)
+        ms = [m0] + [tl3.encode(W) for _ in range(copies - 1)]
+        for m in ms:
+            m.upload()
+        dense = [torch.from_numpy(W).cuda() for _ in range(min(copies, max(2, int(np.ceil(3 * 126e6 / W.nbytes)))))]
+        Xd = torch.from_numpy(case.make_X()).cuda()
+        ws = m0.new_workspace(case.N)
+        Y = torch.empty((case.M, case.N), dtype=torch.float16, device="cuda")
+
+        def ours():
+            for m in ms:
+                m.spmm(Xd, Y, workspace=ws)
+
+        def cublas():
+            for d in dense:
+                torch.matmul(d, Xd, out=Y)
+
+        us = _time_graph(ours) / len(ms)
+        dus = _time_graph(cublas) / len(dense)
+        assert m0.status(ws) == tl3.OK
+        nbytes = m0.device_bytes() + case.K * case.N * 2 + case.M * case.N * 2
+        st = m0.stats()
+        print(json.dumps({"sweep": args.sweep, "point": label, "M": case.M, "K": case.K, "N": case.N,
+                          "sparsity": case.sparsity, "us": round(us, 2), "gbs": round(nbytes / us / 1e3, 1),
+                          "frac_measured": round(nbytes / us / 1e3 / peak, 4),
+                          "dense_equiv_tflops": round(2.0 * case.M * case.K * case.N / us / 1e6, 2),
+                          "dense_gemm_us": round(dus, 2), "speedup_vs_dense": round(dus / us, 3),
+                          "bytes_over_dense": round(st["device_bytes"] / (2 * case.M * case.K), 4),
+                          "sf_share": round(st["n_sf"] / st["nnz"], 4), "res_share": round(st["n_res"] / st["nnz"], 4)}), flush=True)
+        for m in ms:
+            m.close()
+        del dense, Xd, Y, ws
+        torch.cuda.empty_cache()
+
+    if args.sweep == "n":
+        for N in (8, 16, 32, 64, 128, 256, 512):
+            point(wl.Case(4, "n_sweep", 9216, 9216, N, 4000, 0.5, "row_scaled"), f"N={N}")
+    elif args.sweep == "sparsity":
+        for case in wl.config_cases(3):
+            point(case, case.name)
+    elif args.sweep == "stack":
+        cases = list(wl.config_cases(5))
+        ms, dense, Xs, Ys, wss = [], [], [], [], []
+        for c in cases:
+            W = c.make_W()
+            m = tl3.encode(W)
+            m.upload()
+            ms.append(m)
+            dense.append(torch.from_numpy(W).cuda())
+            Xs.append(torch.from_numpy(c.make_X()).cuda())
+            Ys.append(torch.empty((c.M, c.N), dtype=torch.float16, device="cuda"))
+            wss.append(m.new_workspace(c.N))
+
+        def ours():
+            for m, X, Y, ws in zip(ms, Xs, Ys, wss):
+                m.spmm(X, Y, workspace=ws)
+
+        def cublas():
+            for d, X, Y in zip(dense, Xs, Ys):
+                torch.matmul(d, X, out=Y)
+
+        us, dus = _time_graph(ours), _time_graph(cublas)
+        flops = sum(2.0 * c.M * c.K * c.N for c in cases)
+        nbytes = sum(m.device_bytes() + c.K * c.N * 2 + c.M * c.N * 2 for m, c in zip(ms, cases))
+        print(json.dumps({"sweep": "stack", "layers": [f"{c.M}x{c.K}" for c in cases], "N": 16, "us": round(us, 2),
+                          "gbs": round(nbytes / us / 1e3, 1), "frac_measured": round(nbytes / us / 1e3 / peak, 4),
+                          "dense_equiv_tflops": round(flops / us / 1e6, 2), "dense_stack_us": round(dus, 2),
+                          "speedup_vs_dense": round(dus / us, 3),
+                          "res_share": [round(m.stats()["n_res"] / m.stats()["nnz"], 4) for m in ms]}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -414,10 +520,14 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--single", type=int, nargs=3, metavar=("M", "K", "N"), help="run a few launches of one shape and exit")
     ap.add_argument("--launches", type=int, default=3)
+    ap.add_argument("--sweep", choices=["n", "sparsity", "stack"], help="extra measurements; one JSON line per point")
     ap.add_argument("--sparsity", type=float, default=0.5)
     args = ap.parse_args()
     if args.single:
         run_single(args)
+        return
+    if args.sweep:
+        run_sweep(args)
         return
     rank, local_rank, world = dist.env_world()
     if args.impl == "reference":

@@ -126,11 +126,14 @@ int tl3_workspace_init(void* workspace, size_t bytes, void* stream);
  * folded into the same accumulators, one final reduction).
  *   X: device, fp16, K x N row-major, leading dimension ldx >= N, ldx % 8 == 0, 16-byte aligned.
  *   Y: device, fp16, M x N row-major, leading dimension ldy >= N; fully overwritten.
- *   1 <= N <= 64.  fp32 accumulation, fp16 round-to-nearest-even output.  W and X are assumed
- *   finite (an empty slot multiplies an exact zero with an element of X).
+ *   1 <= N <= TL3_MAX_N.  Up to 64 columns are one kernel launch (the decode-phase case the
+ *   kernels are built for); wider blocks are processed 64 columns at a time, each streaming W
+ *   again.  fp32 accumulation, fp16 round-to-nearest-even output.  W and X are assumed finite (an
+ *   empty slot multiplies an exact zero with an element of X).
  * Asynchronous on `stream`; allocates nothing; does not synchronise.  Calls that share a
  * workspace must not overlap on the GPU.
  * Errors: NOT_UPLOADED, INVALID_ARG, UNSUPPORTED (N out of range, device is not sm_100), CUDA. */
+#define TL3_MAX_N 4096
 int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N,
              void* workspace, void* stream);
 

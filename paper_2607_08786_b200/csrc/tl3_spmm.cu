@@ -843,7 +843,7 @@ int tl3_upload(tl3_matrix* m, void* dptr, void* stream) {
 }
 
 size_t tl3_workspace_bytes(const tl3_matrix* m, int N) {
-  if (!m || N < 1 || N > 64) return 0;
+  if (!m || N < 1 || N > TL3_MAX_N) return 0;
   tl3::DeviceInfo di;
   if (tl3::device_info(&di) != TL3_OK) return 0;
   return tl3::workspace_layout(m, tl3::n_pad_of(N), di.sm_count).total;
@@ -855,10 +855,9 @@ int tl3_workspace_init(void* workspace, size_t bytes, void* stream) {
   return TL3_OK;
 }
 
-int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N, void* workspace, void* stream) {
+// one launch: at most 64 columns
+static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N, void* workspace, void* stream) {
   using namespace tl3;
-  if (!m || !X || !Y || !workspace) return TL3_ERR_INVALID_ARG;
-  if (!m->dptr) return TL3_ERR_NOT_UPLOADED;
   if (N < 1 || N > 64) return TL3_ERR_UNSUPPORTED;
   if (ldx < N || ldy < N || (ldx & 7) != 0 || (reinterpret_cast<uintptr_t>(X) & 15) != 0 ||
       (reinterpret_cast<uintptr_t>(Y) & 1) != 0 || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0)
@@ -926,9 +925,25 @@ int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t l
   }
 }
 
+int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N, void* workspace, void* stream) {
+  if (!m || !X || !Y || !workspace) return TL3_ERR_INVALID_ARG;
+  if (!m->dptr) return TL3_ERR_NOT_UPLOADED;
+  if (N < 1 || N > TL3_MAX_N) return TL3_ERR_UNSUPPORTED;
+  if (ldx < N || ldy < N) return TL3_ERR_INVALID_ARG;
+  // Wider activation blocks are processed 64 columns at a time; every block streams W again, so
+  // beyond N = 64 the time grows in proportion to N (this kernel targets the decode phase; the
+  // paper, too, loses to the dense GEMM at large N, Sec. 6).
+  for (int n0 = 0; n0 < N; n0 += 64) {
+    const int nb = N - n0 < 64 ? N - n0 : 64;
+    const int rc = spmm_block(m, static_cast<const uint16_t*>(X) + n0, ldx, static_cast<uint16_t*>(Y) + n0, ldy, nb, workspace, stream);
+    if (rc != TL3_OK) return rc;
+  }
+  return TL3_OK;
+}
+
 int tl3_spmm_host(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int N, void* dX, void* dY, void* workspace, void* stream) {
   if (!m || !X || !Y || !dX || !dY) return TL3_ERR_INVALID_ARG;
-  if (N < 1 || N > 64) return TL3_ERR_UNSUPPORTED;
+  if (N < 1 || N > TL3_MAX_N) return TL3_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // device copy of X with a leading dimension that satisfies the 16-byte rule
   const int64_t ldx = (N + 7) / 8 * 8;
@@ -967,7 +982,7 @@ static int static_scratch_address(void** out) {
 int tl3_spmm_static_scratch(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N, void* stream) {
   if (!m || !X || !Y) return TL3_ERR_INVALID_ARG;
   if (!m->dptr) return TL3_ERR_NOT_UPLOADED;
-  if (N < 1 || N > 64) return TL3_ERR_UNSUPPORTED;
+  if (N < 1 || N > TL3_MAX_N) return TL3_ERR_UNSUPPORTED;
   tl3::DeviceInfo di;
   if (int rc = tl3::device_info(&di)) return rc;
   const tl3::WorkspaceLayout wl = tl3::workspace_layout(m, tl3::n_pad_of(N), di.sm_count);

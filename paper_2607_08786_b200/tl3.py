@@ -234,7 +234,7 @@ class Matrix:
         if Y is None:
             Y = torch.empty((M, N), dtype=torch.float16, device=X.device)
         if workspace is None:
-            key = 16 if N <= 16 else 32 if N <= 32 else 64
+            key = 16 if N <= 16 else 32 if N <= 32 else 64        # wider blocks reuse the 64-column scratch
             workspace = self._workspaces.get(key)
             if workspace is None:
                 workspace = self._workspaces[key] = self.new_workspace(N, stream)

@@ -208,6 +208,15 @@ def test_small_integers_are_exact(tl3, oracle_mod):
     assert np.array_equal(Y.view(np.uint16), oracle_mod.spmm(oracle_mod.encode(W), X))
 
 
+@pytest.mark.parametrize("N", [72, 128, 200])
+def test_wide_activation_blocks(tl3, oracle_mod, N):
+    """N > 64 (towards prefill) runs as 64-column blocks."""
+    case = wl.Case(0, "wide_n", 512, 768, N, 60 + N, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    Y, _ = run_gpu(tl3, W, X, repeats=2)
+    check(oracle_mod, W, X, Y)
+
+
 def test_strided_operands(tl3, oracle_mod):
     case = wl.Case(0, "ld", 300, 700, 12, 5, 0.5, "magnitude")
     W, X = case.make_W(), case.make_X()
@@ -226,7 +235,8 @@ def test_argument_errors_on_device(tl3):
     assert L.tl3_spmm(m._h, X.data_ptr(), 8, Y.data_ptr(), 8, 8, ws.data_ptr(), None) == tl3.ERR_NOT_UPLOADED
     m.upload()
     ws = m.new_workspace(8)
-    assert L.tl3_spmm(m._h, X.data_ptr(), 8, Y.data_ptr(), 8, 65, ws.data_ptr(), None) == tl3.ERR_UNSUPPORTED
+    assert L.tl3_spmm(m._h, X.data_ptr(), 8, Y.data_ptr(), 8, 4097, ws.data_ptr(), None) == tl3.ERR_UNSUPPORTED
+    assert L.tl3_spmm(m._h, X.data_ptr(), 8, Y.data_ptr(), 8, 65, ws.data_ptr(), None) == tl3.ERR_INVALID_ARG   # ldx < N
     assert L.tl3_spmm(m._h, X.data_ptr(), 8, Y.data_ptr(), 8, 0, ws.data_ptr(), None) == tl3.ERR_UNSUPPORTED
     assert L.tl3_spmm(m._h, X.data_ptr(), 12, Y.data_ptr(), 8, 8, ws.data_ptr(), None) == tl3.ERR_INVALID_ARG   # ldx % 8
     assert L.tl3_spmm(m._h, X.data_ptr() + 2, 8, Y.data_ptr(), 8, 8, ws.data_ptr(), None) == tl3.ERR_INVALID_ARG  # X alignment

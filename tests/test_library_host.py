@@ -137,7 +137,7 @@ def test_error_codes(tl3):
     assert L.tl3_pack(m._h, W.ctypes.data, 1 << 20) == tl3.ERR_UNSUPPORTED
     assert L.tl3_spmm(m._h, 16, 8, 16, 8, 8, 256, None) == tl3.ERR_NOT_UPLOADED
     assert L.tl3_spmm(None, None, 8, None, 8, 8, None, None) == tl3.ERR_INVALID_ARG
-    assert L.tl3_workspace_bytes(m._h, 65) == 0 and L.tl3_workspace_bytes(m._h, 0) == 0
+    assert L.tl3_workspace_bytes(m._h, 4097) == 0 and L.tl3_workspace_bytes(m._h, 0) == 0
     assert b"invalid" in L.tl3_strerror(tl3.ERR_INVALID_ARG)
     assert L.tl3_strerror(-99) == b"unknown error"
 
