@@ -277,12 +277,16 @@ __device__ __forceinline__ void sts_zero16B(uint32_t addr) {
   asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
 }
 
-// Algorithm 1 for one chain, eight delta bytes at a time.  `pos` carries offset_t in its low and
+// Algorithm 1 for one chain, one code word (four delta bytes) at a time.  `pos` carries offset_t in its low and
 // offset_r in its high 16 bits, so one add advances both cursors and one shift/xor pair forms both
-// swizzled byte offsets.  Within a batch all positions are formed first, then all W_t loads are
+// swizzled byte offsets.  Within a round all positions are formed first, then all W_t loads are
 // issued, then all stores, so that the shared-memory round trips of different entries overlap; the
-// code words of the next batch are fetched before the current one is processed.
-constexpr int kBatch = 8;
+// next code word is fetched before the current one is processed.  (Longer rounds measured slower:
+// lanes whose chain has ended only execute predicated-off instructions.)
+#ifndef TL3_DECODE_BATCH
+#define TL3_DECODE_BATCH 4
+#endif
+constexpr int kBatch = TL3_DECODE_BATCH;                  // 1, 2 or 4 delta bytes per round of loads and stores
 
 // packed byte offsets (W_t offset low, W_r offset high) of the packed positions `pos`
 __device__ __forceinline__ uint32_t swizzled_offset2(uint32_t pos) { return (pos << 1) ^ ((pos >> 2) & 0x00700070u); }
@@ -295,8 +299,8 @@ __device__ __forceinline__ void decode_chain(uint32_t stage, uint32_t wr, uint32
   uint32_t pos = hdr;
   uint32_t word_addr = code_addr & ~3u;
   const uint32_t shift = (code_addr & 3u) * 8u;
-  uint32_t w0 = 0, w1 = 0, w2 = 0;
-  if (len != 0) { w0 = lds_u32(word_addr); w1 = lds_u32(word_addr + 4); w2 = lds_u32(word_addr + 8); }
+  uint32_t w0 = 0, w1 = 0;
+  if (len != 0) { w0 = lds_u32(word_addr); w1 = lds_u32(word_addr + 4); }
   {                                                     // first pair: absolute 16-bit positions
     const uint32_t off2 = swizzled_offset2(pos);
     const uint32_t at = stage + (off2 & 0xFFFFu);
@@ -304,33 +308,41 @@ __device__ __forceinline__ void decode_chain(uint32_t stage, uint32_t wr, uint32
     sts_u16(at, 0);                                     // W_t[offset_t] = 0
     sts_u16(wr + (off2 >> 16), v);                      // W_r[offset_r] = W_t[offset_t]
   }
-  for (uint32_t k0 = 0; k0 < len; k0 += kBatch) {
-    uint32_t lo = __funnelshift_r(w0, w1, shift), hi = __funnelshift_r(w1, w2, shift);
+  for (uint32_t k0 = 0; k0 < len; k0 += 4) {            // four delta bytes = one (unaligned) code word
+    uint32_t bytes = __funnelshift_r(w0, w1, shift);
     const uint32_t rem = len - k0;
-    if (rem > kBatch) {                                 // code words of the next batch
-      word_addr += kBatch;
-      w0 = w2; w1 = lds_u32(word_addr + 4); w2 = lds_u32(word_addr + 8);
-    } else if (rem < kBatch) {                          // bytes past the end behave like dummies
-      if (rem <= 4) { hi = 0; if (rem < 4) lo &= (1u << (8 * rem)) - 1u; }
-      else hi &= (1u << (8 * (rem - 4))) - 1u;
-    }
-    uint32_t off2[kBatch], val[kBatch];
-    bool real[kBatch];
-#pragma unroll
-    for (int q = 0; q < kBatch; ++q) {
-      const uint32_t bt = __byte_perm(q < 4 ? lo : hi, 0u, 0x4440u + (q & 3));   // delta byte q
-      const uint32_t delta = (bt * 0x1001u) & 0x000F000Fu;      // t delta | r delta << 16
-      pos += delta;
-      real[q] = ((delta - 0x00010001u) & 0x80008000u) == 0u;    // both nibbles non-zero (else a dummy point)
-      if (pos & 0xE000E000u) { real[q] = false; *bad = 2u; }
-      off2[q] = swizzled_offset2(pos);
+    if (rem > 4) {                                      // code word of the next round
+      word_addr += 4;
+      w0 = w1;
+      w1 = lds_u32(word_addr + 4);
+    } else if (rem < 4) {                               // bytes past the end behave like dummies
+      bytes &= (1u << (8 * rem)) - 1u;
     }
 #pragma unroll
-    for (int q = 0; q < kBatch; ++q)
-      if (real[q]) val[q] = lds_u16(stage + (off2[q] & 0xFFFFu));
+    for (int b0 = 0; b0 < 4; b0 += kBatch) {
+      uint32_t off2[kBatch], val[kBatch];
+      bool real[kBatch];
 #pragma unroll
-    for (int q = 0; q < kBatch; ++q)
-      if (real[q]) { sts_u16(stage + (off2[q] & 0xFFFFu), 0); sts_u16(wr + (off2[q] >> 16), val[q]); }
+      for (int q = 0; q < kBatch; ++q) {
+        const uint32_t bt = __byte_perm(bytes, 0u, 0x4440u + b0 + q);   // delta byte b0 + q
+        const uint32_t delta = (bt * 0x1001u) & 0x000F000Fu;      // t delta | r delta << 16
+        pos += delta;
+        real[q] = ((delta - 0x00010001u) & 0x80008000u) == 0u;    // both nibbles non-zero (else a dummy point)
+        off2[q] = swizzled_offset2(pos);
+      }
+      // both cursors only grow, so the last position of the round bounds them all
+      if (pos & 0xE000E000u) {
+        *bad = 2u;
+#pragma unroll
+        for (int q = 0; q < kBatch; ++q) real[q] = false;
+      }
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q)
+        if (real[q]) val[q] = lds_u16(stage + (off2[q] & 0xFFFFu));
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q)
+        if (real[q]) { sts_u16(stage + (off2[q] & 0xFFFFu), 0); sts_u16(wr + (off2[q] >> 16), val[q]); }
+    }
   }
 }
 
@@ -868,8 +880,8 @@ static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, 
   const int n_pad = n_pad_of(N);
 
   // shared-memory plan
-  // + 16: the decoder fetches delta bytes in aligned words and may read a few bytes past a block
-  const uint32_t block_area = (m->max_block_bytes + 16u + 1023u) / 1024u * 1024u;
+  // + 48: the decoder fetches delta bytes in aligned words, one batch ahead, and may read that far past a block
+  const uint32_t block_area = (m->max_block_bytes + 48u + 1023u) / 1024u * 1024u;
   const uint32_t x_bytes = 128u * n_pad * 2u;
   const uint32_t stage_stride = block_area + x_bytes;
   const uint32_t fixed = kWrBuffers * kWrBytes + kBarrierBytes + 1024u;   // + alignment slack
