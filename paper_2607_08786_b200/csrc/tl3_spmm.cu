@@ -60,10 +60,10 @@ constexpr int kEpilogueWarp0 = kDecodeWarp0 + 4 * kGroups;
 constexpr int kThreads = (kEpilogueWarp0 + 4) * 32;
 constexpr int kMaxStages = 8;
 constexpr uint32_t kWrBytes = 16384;
-constexpr int kWrBuffers = 4;             // W_r ring: tile i uses buffer i % 4
+constexpr int kMaxWrBuffers = 5;          // W_r ring: tile i uses buffer i % num_wr (4 or 5, as shared memory allows)
 constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColMetaT = 128;       // + 4 * (tile % 4): metadata of W_t, four columns per tile in flight
-constexpr uint32_t kColMetaR = 144;       // two columns of 0xEEEEEEEE
+constexpr uint32_t kColMetaT = 128;       // + 4 * (W_r buffer): metadata of W_t, four columns per tile in flight
+constexpr uint32_t kColMetaR = 152;       // two columns of 0xEEEEEEEE
 constexpr uint32_t kSmemLimit = 232448;   // 227 KB
 constexpr uint32_t kBarrierBytes = 1024;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per kernel
@@ -93,6 +93,7 @@ struct KernelArgs {
   uint32_t stage_stride;     // bytes per stage (block area + X tile), multiple of 1024
   uint32_t x_offset;         // offset of the X tile inside a stage, multiple of 1024
   int num_stages;
+  int num_wr;                // W_r buffers (4 or 5)
   long long* timing;         // phase-timing buffer (debug builds), else null
 };
 
@@ -352,12 +353,13 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int S = a.num_stages;
-  uint8_t* wr_base = smem + static_cast<size_t>(S) * a.stage_stride;           // kWrBuffers x 16 KB
-  uint8_t* bar_base = wr_base + kWrBuffers * kWrBytes;
-  // barrier block: full[8] mma_done[8] decoded[8] acc_full[2] acc_empty[2] wr_ready[4] | tmem slot | flags | wr_free[4]
+  const int NW = a.num_wr;
+  uint8_t* wr_base = smem + static_cast<size_t>(S) * a.stage_stride;           // NW x 16 KB
+  uint8_t* bar_base = wr_base + NW * kWrBytes;
+  // barrier block: full[8] mma_done[8] decoded[8] acc_full[2] acc_empty[2] | tmem slot | flags | wr_ready[5] wr_free[5]
   uint64_t* bars = reinterpret_cast<uint64_t*>(bar_base);
   const uint32_t bar_full = smem_u32(bars), bar_mma = smem_u32(bars + 8), bar_dec = smem_u32(bars + 16);
-  const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26), bar_wrready = smem_u32(bars + 28), bar_wrfree = smem_u32(bars + 36);
+  const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26), bar_wrready = smem_u32(bars + 44), bar_wrfree = smem_u32(bars + 49);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 32);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 33);
   volatile unsigned int* last_flag = reinterpret_cast<volatile unsigned int*>(bars + 34);
@@ -369,7 +371,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   const int kt_begin = static_cast<int>(t_begin % a.tiles_k);
   // Decode groups in use: a group may wait for its next tile only once the stage's previous
   // phase has completed (a parity wait cannot tell phases two apart), which holds as long as
-  // there are no more groups than stages.  Tile i goes to group i % AG and W_r buffer i % AG.
+  // there are no more groups than stages.  Tile i goes to group i % AG and W_r buffer i % NW.
   const int AG = S < kGroups ? S : kGroups;
   const uint32_t smem_base = smem_u32(smem);
 
@@ -383,7 +385,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       mbar_init(bar_accfull + 8 * b, 1);
       mbar_init(bar_accempty + 8 * b, 128);
     }
-    for (int w = 0; w < kWrBuffers; ++w) { mbar_init(bar_wrready + 8 * w, 64); mbar_init(bar_wrfree + 8 * w, 1); }
+    for (int w = 0; w < kMaxWrBuffers; ++w) { mbar_init(bar_wrready + 8 * w, 64); mbar_init(bar_wrfree + 8 * w, 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -466,8 +468,8 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     }
   } else if (warp == kClearWarp0 || warp == kClearWarp0 + 1) {
     // ------------------------------------------------------------------ W_r clearing
-    // Tile i scatters into W_r buffer i % AG.  These two warps zero a buffer as soon as the MMAs
-    // of tile i - AG (its previous user) are done (the MMA warp commits to the buffer's own
+    // Tile i scatters into W_r buffer i % NW.  These two warps zero a buffer as soon as the MMAs
+    // of tile i - NW (its previous user) are done (the MMA warp commits to the buffer's own
     // barrier) and then open it for the decode warps, so the decode path neither clears nor needs
     // a group-wide barrier.
     const int ct = tid - kClearWarp0 * 32;                       // 0..63
@@ -482,7 +484,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       for (int c = 0; c < 16; ++c) sts_zero16B(wr + (c * 64 + ct) * 16);
       fence_proxy_async_smem();                                  // the MMA reads what stays zero
       mbar_arrive(bar_wrready + 8 * wb);
-      if (++wb == AG) { wb = 0; ++use; }
+      if (++wb == NW) { wb = 0; ++use; }
     }
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
@@ -539,7 +541,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       a_lo += stride16;
       if (++s == S) { s = 0; ph ^= 1u; a_lo = a_lo0; }
       if (++kt == a.tiles_k) kt = 0;
-      if (++wb == AG) wb = 0;
+      if (++wb == NW) wb = 0;
     }
     if (lane == 0) TL3_TDUMP(8)
   } else if (warp >= kDecodeWarp0 && warp < kEpilogueWarp0) {
@@ -552,9 +554,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};"
                    ::"r"(tmem_base + lane_base + kColMetaR), "r"(0xEEEEEEEEu), "r"(0xEEEEEEEEu) : "memory");
     }
-    static_assert(kWrBuffers == kGroups, "group g owns W_r buffer g");
-    const int wb = g;                                           // this group's W_r buffer and metadata columns
-    const uint32_t wr = wr0 + wb * kWrBytes;
+    int wb = g % NW, use = g / NW;                              // W_r buffer of tile i and how often it was filled before
     int s = g;                                                  // g < AG <= S
     uint32_t ph = 0;
     TL3_T0()
@@ -564,12 +564,13 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       // first, so the four warps get blocks of different length; the block a warp takes rotates
       // from tile to tile to even the load out.
       const int cr = (r + 32 * (j & 3)) & 127;                  // chain handled by this thread
+      const uint32_t wr = wr0 + wb * kWrBytes;
       // Order matters.  The W_r buffer is ready once the MMAs of tile i - AG are done, and MMAs
       // are issued in tile order, so by then every tile up to i - AG -- in particular the previous
       // user of this stage, tile i - S -- has been loaded and consumed.  Only then is the parity
       // wait on the stage's `full` barrier unambiguous (loads may complete out of order, and a
       // parity wait cannot tell "two phases back" from "done").
-      bool ok = mbar_wait(bar_wrready + 8 * wb, j & 1, wctx, kStDecodeWrReady);
+      bool ok = mbar_wait(bar_wrready + 8 * wb, use & 1, wctx, kStDecodeWrReady);
       TL3_TACC(1)
       ok = ok && mbar_wait(bar_full + 8 * s, ph, wctx, kStDecodeFull);
       TL3_TACC(2)
@@ -633,6 +634,8 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       TL3_TACC(7)
       s += AG;
       while (s >= S) { s -= S; ph ^= 1u; }
+      wb += AG;
+      while (wb >= NW) { wb -= NW; ++use; }
     }
     if (lane == 0) TL3_TDUMP(16 + 8 * (warp - kDecodeWarp0))
   } else if (warp >= kEpilogueWarp0) {
@@ -884,10 +887,17 @@ static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, 
   const uint32_t block_area = (m->max_block_bytes + 48u + 1023u) / 1024u * 1024u;
   const uint32_t x_bytes = 128u * n_pad * 2u;
   const uint32_t stage_stride = block_area + x_bytes;
-  const uint32_t fixed = kWrBuffers * kWrBytes + kBarrierBytes + 1024u;   // + alignment slack
-  if (fixed + 2u * stage_stride > kSmemLimit) return TL3_ERR_UNSUPPORTED;
-  int stages = static_cast<int>((kSmemLimit - fixed) / stage_stride);
+  // W_r ring of five buffers if that still leaves five stages, else four
+  int num_wr = kMaxWrBuffers, stages = 0;
+  uint32_t fixed = 0;
+  for (;; --num_wr) {
+    fixed = num_wr * kWrBytes + kBarrierBytes + 1024u;          // + alignment slack
+    stages = fixed + stage_stride <= kSmemLimit ? static_cast<int>((kSmemLimit - fixed) / stage_stride) : 0;
+    if (stages >= 5 || num_wr == 4) break;
+  }
+  if (stages < 2) return TL3_ERR_UNSUPPORTED;
   if (stages > kMaxStages) stages = kMaxStages;
+  if (num_wr == kMaxWrBuffers && stages > 5) stages = 5;        // a sixth stage measured no faster than five
   const uint32_t smem_bytes = fixed + static_cast<uint32_t>(stages) * stage_stride;
 
   // tensor map of X: dims {N, K}, box {n_pad, 128}; columns >= N and rows >= K read as zero
@@ -923,6 +933,7 @@ static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, 
   args.stage_stride = stage_stride;
   args.x_offset = block_area;
   args.num_stages = stages;
+  args.num_wr = num_wr;
 #ifdef TL3_PHASE_TIMING
   args.timing = g_timing_buffer;
 #else
