@@ -389,6 +389,13 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // the producer's first directory entries and the X tensor map: start the (cold) global fetches
+  // before the set-up barrier
+  uint4 dir_first = make_uint4(0, 0, 0, 0);
+  if (warp == kProducerWarp) {
+    if (lane < n_tiles) dir_first = __ldg(reinterpret_cast<const uint4*>(a.dir + t_begin + lane));
+    if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
+  }
   if (warp == kAllocWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -413,8 +420,11 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     const int pre = n_tiles < S ? n_tiles : S;                  // tiles whose stages are free at the start
     TL3_T0()
     for (int base = 0; base < n_tiles && alive; base += 32) {
-      uint4 mine = make_uint4(0, 0, 0, 0);
-      if (base + lane < n_tiles) mine = __ldg(reinterpret_cast<const uint4*>(a.dir + t_begin + base + lane));
+      uint4 mine = dir_first;
+      if (base > 0) {
+        mine = make_uint4(0, 0, 0, 0);
+        if (base + lane < n_tiles) mine = __ldg(reinterpret_cast<const uint4*>(a.dir + t_begin + base + lane));
+      }
       const int cnt = n_tiles - base < 32 ? n_tiles - base : 32;
       if (base == 0) {
         for (int j = 0; j < pre; ++j) {                          // S <= 8 < 32: all in this batch
