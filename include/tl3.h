@@ -98,14 +98,18 @@ void tl3_free(tl3_matrix* m);
 
 /* ---- device side (Sec. 4) -------------------------------------------------------------- */
 
-/* Size of the packed device blob (tile blocks ready for bulk copies). */
+/* Size of the packed device blob (tile blocks ready for bulk copies); 0 for a container whose
+ * tiles are not 128 x 128 (the device path exists for that tile only). */
 size_t tl3_device_bytes(const tl3_matrix* m);
 
 /* Pack the container into a HOST buffer of tl3_device_bytes() bytes: exactly the bytes tl3_upload()
- * sends to the device (a permutation of the canonical arrays plus alignment padding: per tile one
- * contiguous block holding the value slots in the shared-memory image the MMA reads, the metadata
- * in tensor-memory word order, the chain starts, lengths and delta bytes, and the Residual
- * entries).  For callers that stage the blob themselves.  Errors: UNSUPPORTED, INVALID_ARG. */
+ * sends to the device: per tile one contiguous block holding the value slots in the shared-memory
+ * image the MMA reads, the metadata in tensor-memory word order, the chain starts, lengths and delta
+ * bytes, and the Residual entries.  Values, metadata and the sets of parked and Residual elements
+ * are those of the canonical container; which empty slot a parked element sits in and how the
+ * PDD chains are cut follow the banks of shared memory (Sec. 3.2 leaves both open), so the PDD
+ * bytes differ from the canonical ones.  For callers that stage the blob themselves.
+ * Errors: UNSUPPORTED, INVALID_ARG. */
 int tl3_pack(const tl3_matrix* m, void* host_buf, size_t bytes);
 
 /* Pack the container and copy it to dptr (device, >= tl3_device_bytes(), 256-byte aligned) on

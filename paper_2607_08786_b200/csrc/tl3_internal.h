@@ -27,6 +27,7 @@ struct tl3_matrix {
   void* dptr = nullptr;
   size_t device_bytes = 0;             // computed lazily by tl3_device_bytes
   uint32_t max_block_bytes = 0;
+  std::vector<uint32_t> dev_sizes;     // per tile: PDD bytes and Residual entries of the device image
   size_t dir_offset = 0, blocks_offset = 0;
 
   // last launch geometry
@@ -42,16 +43,19 @@ namespace tl3 {
 //
 // Tile block (tile 128 x 128, H = 64 value slots per row):
 //   +0      values   128 rows x 128 B, the K-major 128-byte-swizzled image the MMA descriptor
-//                    reads: 16-byte chunk j of row r sits at chunk (j ^ (r & 7))
+//                    reads: 16-byte chunk j of row r sits at chunk (j ^ (r & 7)).  Kept values are
+//                    those of the canonical container; parked values are re-parked bank-major
+//                    (see tl3_pack.cpp)
 //   +16384  metadata 128 x 16 B: word kb of entry L is the TMEM word of lane L for k-block kb:
 //                    bits 0-15 = nibbles of windows 8kb+4h .. 8kb+4h+3 of row (L&7)+16(L>>4),
 //                    bits 16-31 = the same windows of that row + 8, with h = (L>>3)&1
 //   +18432  u32[4]: pdd_len, res_cnt, 0, 0
-//   +18448  chain starts u32[128]: tau0 | rho0 << 16 (0xFFFFFFFF = empty chain), chains sorted
-//           longest first (ties: lower row first)
+//   +18448  chain starts u32[128]: tau0 | rho0 << 16 (0xFFFFFFFF = empty chain) in the bank-major
+//           slot coordinate u = bank << 8 | slot-in-window << 7 | row; chain slot w * 32 + l holds
+//           the w-th longest of the four chains whose empty slots lie in bank l
 //   +18960  chain lengths u8[128], same order
 //   +19088  PDD delta bytes, chain after chain in that order, padded to 4 bytes
-//   +...    Residual entries u32[res_cnt]: rho | value << 16, padded to 16 bytes
+//   +...    Residual entries u32[res_cnt]: u of the element | value << 16, padded to 16 bytes
 constexpr int kTileM = 128, kTileK = 128, kH = 64;
 constexpr uint32_t kValsBytes = 16384, kMetaOff = 16384, kMetaBytes = 2048;
 constexpr uint32_t kInfoOff = 18432, kHdrOff = 18448, kLenOff = 18960, kPddOff = 19088;

@@ -1,8 +1,24 @@
-// Device packer: lays the canonical container out as one blob of per-tile blocks, each ready for
-// a single bulk copy into shared memory (layout described in tl3_internal.h).  The blob is a
-// permutation of the canonical bytes plus alignment padding; nothing is re-encoded.
+// Device packer: turns the canonical container into one blob of per-tile blocks, each ready for a
+// single bulk copy into shared memory (layout described in tl3_internal.h).
+//
+// Values and metadata are carried over unchanged (permuted into the image the MMA reads).  The
+// Slot-Filling layer is re-paired and its PDD chains re-cut for the 32 banks of shared memory:
+// the canonical container pairs the i-th surplus element with the i-th empty slot in row-major
+// order and cuts one chain per tile row, which makes the 32 lanes of a decode warp touch random
+// banks.  Here both streams are ordered bank-major -- a slot's coordinate is
+//     u = bank << 8 | slot-in-window << 7 | row,      bank = word of the 128-byte swizzled row
+// -- the i-th surplus element in that order is parked in the i-th selected empty slot in that
+// order, and chain c holds the pairs whose empty slot has u >> 6 == c.  Lane l of a decode warp
+// takes a chain of bank l, so its loads and stores in W_t never collide with another lane's, and
+// its stores in W_r land in bank l or a neighbour.  It is the same format (Sec. 3.2: values parked
+// in empty slots, 16-bit absolute starts, 4-bit delta pairs, dummy points, Residual list) over a
+// different enumeration of the tile's slots; the set of parked elements, the set of Residual
+// elements and all values are those of the canonical container.
 #include <algorithm>
+#include <atomic>
 #include <cstring>
+#include <thread>
+#include <vector>
 
 #include "tl3_internal.h"
 
@@ -14,8 +30,171 @@ static inline uint32_t block_bytes(uint32_t pdd_len, uint32_t res_cnt) {
   return align_up(kPddOff + align_up(pdd_len, 4) + 4 * res_cnt, 16);
 }
 
+// slot position pos = row * 64 + 2 * window + slot-in-window  <->  bank-major coordinate u
+static inline uint32_t u_of_pos(uint32_t pos) {
+  const uint32_t r = pos >> 6, q = (pos >> 1) & 31u, s = pos & 1u;
+  const uint32_t bank = (((q >> 2) ^ (r & 7u)) << 2) | (q & 3u);
+  return (bank << 8) | (s << 7) | r;
+}
+static inline uint32_t pos_of_u(uint32_t u) {
+  const uint32_t r = u & 127u, s = (u >> 7) & 1u, bank = u >> 8;
+  const uint32_t q = (((bank >> 2) ^ (r & 7u)) << 2) | (bank & 3u);
+  return r * 64u + 2u * q + s;
+}
+// byte offset of slot u in the 128-byte-swizzled K-major image (row pitch 128 B)
+static inline uint32_t image_offset(uint32_t u) { return ((u & 127u) << 7) | ((u >> 6) & 0x7Eu); }
+
+namespace {
+
+constexpr int kSlots = kTileM * kH;      // 8192
+constexpr int kChains = 128;             // u >> 6
+
+struct TileCode {
+  uint32_t pdd_len = 0, res_cnt = 0;
+  uint16_t vals[kSlots];                 // by pos; parked values removed, then re-parked
+  uint32_t hdr[kChains];                 // by chain c (u order): u_tau0 | u_rho0 << 16
+  uint8_t len[kChains];
+  uint32_t code_off[kChains];
+  std::vector<uint8_t> code;             // chain after chain in u order
+  std::vector<uint32_t> res;             // u_rho | value << 16
+};
+
+// Re-pairs and re-chains tile (tm, tk).
+void build_tile(const tl3_matrix* m, int64_t tm, int64_t tk, TileCode& tc) {
+  const int64_t t = tm * m->tiles_k + tk;
+  const int64_t half_ld = m->K_pad / 2;
+  for (int r = 0; r < kTileM; ++r)
+    std::memcpy(&tc.vals[r * kH], &m->tc_vals[(tm * kTileM + r) * half_ld + tk * kH], kH * sizeof(uint16_t));
+  // the parked elements of the canonical chains: value, and where it belongs (by u)
+  static thread_local std::vector<uint16_t> sval(kSlots);
+  static thread_local std::vector<uint8_t> sflag(kSlots);
+  std::fill(sflag.begin(), sflag.end(), 0);
+  uint32_t n_pairs = 0;
+  const uint32_t pdd_off = m->tile_dir[t * 4];
+  uint32_t byte_at = pdd_off;
+  auto take = [&](uint32_t tau, uint32_t rho) {
+    const uint32_t ur = u_of_pos(rho);
+    sval[ur] = tc.vals[tau];
+    sflag[ur] = 1;
+    tc.vals[tau] = 0;
+    ++n_pairs;
+  };
+  for (int r = 0; r < kTileM; ++r) {
+    const uint32_t len = m->chain_len[t * kTileM + r];
+    uint32_t tau = m->chain_tau0[t * kTileM + r], rho = m->chain_rho0[t * kTileM + r];
+    if (tau != 0xFFFFu) {
+      take(tau, rho);
+      for (uint32_t k = 0; k < len; ++k) {
+        const uint32_t b = m->pdd_bytes[byte_at + k], dt = b & 15u, dr = b >> 4;
+        tau += dt;
+        rho += dr;
+        if (dt && dr) take(tau, rho);
+      }
+    }
+    byte_at += len;
+  }
+  // empty slots in u order (every slot whose value is zero: kept values are non-zero), per chain
+  uint32_t cand_count[kChains];
+  uint32_t n_cand = 0;
+  static thread_local std::vector<uint8_t> cand(kSlots);
+  for (int c = 0; c < kChains; ++c) {
+    uint32_t n = 0;
+    for (uint32_t u = 64u * c; u < 64u * c + 64u; ++u) {
+      const bool e = (tc.vals[pos_of_u(u)] & 0x7FFFu) == 0;
+      cand[u] = e;
+      n += e;
+    }
+    cand_count[c] = n;
+    n_cand += n;
+  }
+  // n_pairs <= n_cand (the canonical encoder parked each element in an empty slot).  Chain c
+  // uses the first quota(c) of its empty slots, quotas proportional to what the chain has, so
+  // the parked elements spread evenly over chains however many empty slots stay unused.
+  tc.code.clear();
+  tc.res.clear();
+  uint32_t ur = 0;                        // cursor in the surplus stream
+  auto next_surplus = [&]() { while (!sflag[ur]) ++ur; return ur++; };
+  uint64_t cum = 0;
+  for (int c = 0; c < kChains; ++c) {
+    const uint64_t lo = n_cand ? cum * n_pairs / n_cand : 0;
+    cum += cand_count[c];
+    const uint64_t hi = n_cand ? cum * n_pairs / n_cand : 0;
+    uint32_t quota = static_cast<uint32_t>(hi - lo);
+    tc.hdr[c] = 0xFFFFFFFFu;
+    tc.len[c] = 0;
+    tc.code_off[c] = static_cast<uint32_t>(tc.code.size());
+    uint32_t prev_t = 0, prev_r = 0, n_bytes = 0;
+    bool first = true, overflow = false;
+    for (uint32_t u = 64u * c; quota && u < 64u * c + 64u; ++u) {
+      if (!cand[u]) continue;
+      --quota;
+      const uint32_t r_u = next_surplus();
+      const uint16_t v = sval[r_u];
+      if (overflow) { tc.res.push_back(r_u | static_cast<uint32_t>(v) << 16); continue; }
+      if (first) {
+        tc.hdr[c] = u | r_u << 16;
+        first = false;
+      } else {
+        uint32_t gt = u - prev_t, gr = r_u - prev_r;
+        const uint32_t need = (gt - 1) / 15 + (gr - 1) / 15 + 1;
+        if (n_bytes + need > 255u) {        // a chain holds at most 255 delta bytes: the rest goes to the Residual list
+          overflow = true;
+          tc.res.push_back(r_u | static_cast<uint32_t>(v) << 16);
+          continue;
+        }
+        while (gt > 15) { tc.code.push_back(0x0F); gt -= 15; }     // dummy points (a zero nibble moves nothing)
+        while (gr > 15) { tc.code.push_back(0xF0); gr -= 15; }
+        tc.code.push_back(static_cast<uint8_t>(gt | gr << 4));
+        n_bytes += need;
+      }
+      prev_t = u;
+      prev_r = r_u;
+      tc.vals[pos_of_u(u)] = v;
+    }
+    tc.len[c] = static_cast<uint8_t>(n_bytes);
+  }
+  // canonical Residual entries, in the same coordinate
+  const uint32_t res_off = m->tile_dir[t * 4 + 2], res_cnt = m->tile_dir[t * 4 + 3];
+  for (uint32_t j = 0; j < res_cnt; ++j)
+    tc.res.push_back(u_of_pos(m->res_rho[res_off + j]) | static_cast<uint32_t>(m->res_val[res_off + j]) << 16);
+  for (; ur < static_cast<uint32_t>(kSlots); ++ur)          // none left unless the container had more parked elements than empty slots
+    if (sflag[ur]) tc.res.push_back(ur | static_cast<uint32_t>(sval[ur]) << 16);
+  tc.pdd_len = static_cast<uint32_t>(tc.code.size());
+  tc.res_cnt = static_cast<uint32_t>(tc.res.size());
+}
+
+template <class F>
+void for_each_tile(const tl3_matrix* m, F&& f) {
+  unsigned hw = std::thread::hardware_concurrency();
+  const int n_threads = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(hw ? hw : 1, m->n_tiles / 64 + 1)));
+  std::atomic<int64_t> next{0};
+  auto worker = [&]() {
+    std::vector<TileCode> tc(1);
+    for (;;) {
+      const int64_t t0 = next.fetch_add(16);
+      if (t0 >= m->n_tiles) break;
+      for (int64_t t = t0; t < std::min<int64_t>(t0 + 16, m->n_tiles); ++t) {
+        build_tile(m, t / m->tiles_k, t % m->tiles_k, tc[0]);
+        f(t, tc[0]);
+      }
+    }
+  };
+  std::vector<std::thread> pool;
+  for (int i = 1; i < n_threads; ++i) pool.emplace_back(worker);
+  worker();
+  for (auto& th : pool) th.join();
+}
+
+}  // namespace
+
 size_t plan_device_layout(tl3_matrix* m) {
+  if (m->p.tile_m != kTileM || m->p.tile_k != kTileK) return 0;   // the device image exists for 128 x 128 tiles only
   if (m->device_bytes) return m->device_bytes;
+  m->dev_sizes.assign(static_cast<size_t>(m->n_tiles) * 2, 0);
+  for_each_tile(m, [&](int64_t t, const TileCode& tc) {
+    m->dev_sizes[2 * t] = tc.pdd_len;
+    m->dev_sizes[2 * t + 1] = tc.res_cnt;
+  });
   size_t off = 256;
   m->dir_offset = off;
   off += static_cast<size_t>(m->n_tiles) * sizeof(DirEntry);
@@ -23,7 +202,7 @@ size_t plan_device_layout(tl3_matrix* m) {
   m->blocks_offset = off;
   uint32_t max_block = 0;
   for (int64_t t = 0; t < m->n_tiles; ++t) {
-    const uint32_t b = block_bytes(m->tile_dir[t * 4 + 1], m->tile_dir[t * 4 + 3]);
+    const uint32_t b = block_bytes(m->dev_sizes[2 * t], m->dev_sizes[2 * t + 1]);
     if (b > max_block) max_block = b;
     off += align_up(b, kBlockAlign);
   }
@@ -36,67 +215,60 @@ void pack_device_blob(const tl3_matrix* m, uint8_t* out) {
   std::memset(out, 0, m->device_bytes);
   // header (informational; the kernel takes its geometry from its arguments)
   struct { uint32_t magic, version; int64_t M, K, M_pad, K_pad, n_tiles; uint64_t dir_off, blocks_off; uint32_t max_block; } hdr{
-      0x33334C54u, 1, m->M, m->K, m->M_pad, m->K_pad, m->n_tiles, m->dir_offset, m->blocks_offset, m->max_block_bytes};
+      0x33334C54u, 2, m->M, m->K, m->M_pad, m->K_pad, m->n_tiles, m->dir_offset, m->blocks_offset, m->max_block_bytes};
   std::memcpy(out, &hdr, sizeof(hdr));
   DirEntry* dir = reinterpret_cast<DirEntry*>(out + m->dir_offset);
-  const int64_t half_ld = m->K_pad / 2, meta_ld = m->K_pad / 8;
-  size_t off = m->blocks_offset;
-  for (int64_t tm = 0; tm < m->tiles_m; ++tm) {
-    for (int64_t tk = 0; tk < m->tiles_k; ++tk) {
-      const int64_t t = tm * m->tiles_k + tk;
-      const uint32_t pdd_off = m->tile_dir[t * 4], pdd_len = m->tile_dir[t * 4 + 1];
-      const uint32_t res_off = m->tile_dir[t * 4 + 2], res_cnt = m->tile_dir[t * 4 + 3];
-      const uint32_t bytes = block_bytes(pdd_len, res_cnt);
-      uint8_t* blk = out + off;
-      dir[t] = DirEntry{static_cast<uint32_t>(off / 16), bytes, pdd_len, res_cnt};
-      // values: row r, 16-byte chunk j -> chunk j ^ (r & 7)
-      for (int r = 0; r < kTileM; ++r) {
-        const uint8_t* src = reinterpret_cast<const uint8_t*>(&m->tc_vals[(tm * kTileM + r) * half_ld + tk * kH]);
-        for (int j = 0; j < 8; ++j) std::memcpy(blk + r * 128 + ((j ^ (r & 7)) << 4), src + j * 16, 16);
-      }
-      // metadata in tensor-memory lane order
-      uint32_t* meta = reinterpret_cast<uint32_t*>(blk + kMetaOff);
-      for (int L = 0; L < 128; ++L) {
-        const int row = (L & 7) + 16 * (L >> 4), half = (L >> 3) & 1;
-        for (int kb = 0; kb < 4; ++kb) {
-          // canonical bytes: 2 windows per byte; k-block kb covers windows 8kb..8kb+7 = bytes 4kb..4kb+3
-          const uint8_t* lo = &m->tc_meta[(tm * kTileM + row) * meta_ld + tk * (kTileK / 8) + 4 * kb + 2 * half];
-          const uint8_t* hi = &m->tc_meta[(tm * kTileM + row + 8) * meta_ld + tk * (kTileK / 8) + 4 * kb + 2 * half];
-          meta[L * 4 + kb] = static_cast<uint32_t>(lo[0]) | static_cast<uint32_t>(lo[1]) << 8 |
-                             static_cast<uint32_t>(hi[0]) << 16 | static_cast<uint32_t>(hi[1]) << 24;
-        }
-      }
-      uint32_t* info = reinterpret_cast<uint32_t*>(blk + kInfoOff);
-      info[0] = pdd_len;
-      info[1] = res_cnt;
-      // Chains are stored longest first (ties: lower row first).  A decode thread takes the chain at
-      // its own index, so the 32 lanes of a warp get chains of similar length and few lanes idle
-      // while the longest one finishes.  Which row a chain belongs to is carried by its rho values.
-      int order[kTileM];
-      uint32_t start[kTileM];
-      {
-        uint32_t acc = 0;
-        for (int r = 0; r < kTileM; ++r) { order[r] = r; start[r] = acc; acc += m->chain_len[t * kTileM + r]; }
-        std::stable_sort(order, order + kTileM, [&](int a, int b) {
-          return m->chain_len[t * kTileM + a] > m->chain_len[t * kTileM + b];
-        });
-      }
-      uint32_t* hdrs = reinterpret_cast<uint32_t*>(blk + kHdrOff);
-      uint8_t* code = blk + kPddOff;
-      for (int j = 0; j < kTileM; ++j) {
-        const int r = order[j];
-        const uint32_t len = m->chain_len[t * kTileM + r];
-        hdrs[j] = static_cast<uint32_t>(m->chain_tau0[t * kTileM + r]) | static_cast<uint32_t>(m->chain_rho0[t * kTileM + r]) << 16;
-        blk[kLenOff + j] = static_cast<uint8_t>(len);
-        if (len) std::memcpy(code, &m->pdd_bytes[pdd_off + start[r]], len);
-        code += len;
-      }
-      uint32_t* res = reinterpret_cast<uint32_t*>(blk + kPddOff + align_up(pdd_len, 4));
-      for (uint32_t j = 0; j < res_cnt; ++j)
-        res[j] = static_cast<uint32_t>(m->res_rho[res_off + j]) | static_cast<uint32_t>(m->res_val[res_off + j]) << 16;
-      off += align_up(bytes, kBlockAlign);
+  std::vector<size_t> block_off(static_cast<size_t>(m->n_tiles));
+  {
+    size_t off = m->blocks_offset;
+    for (int64_t t = 0; t < m->n_tiles; ++t) {
+      block_off[t] = off;
+      off += align_up(block_bytes(m->dev_sizes[2 * t], m->dev_sizes[2 * t + 1]), kBlockAlign);
     }
   }
+  const int64_t meta_ld = m->K_pad / 8;
+  for_each_tile(m, [&](int64_t t, const TileCode& tc) {
+    const int64_t tm = t / m->tiles_k, tk = t % m->tiles_k;
+    uint8_t* blk = out + block_off[t];
+    dir[t] = DirEntry{static_cast<uint32_t>(block_off[t] / 16), block_bytes(tc.pdd_len, tc.res_cnt), tc.pdd_len, tc.res_cnt};
+    // values: slot u of the tile at image_offset(u) (row r, 16-byte chunk j -> chunk j ^ (r & 7))
+    for (uint32_t pos = 0; pos < static_cast<uint32_t>(kSlots); ++pos)
+      std::memcpy(blk + image_offset(u_of_pos(pos)), &tc.vals[pos], 2);
+    // metadata in tensor-memory lane order
+    uint32_t* meta = reinterpret_cast<uint32_t*>(blk + kMetaOff);
+    for (int L = 0; L < 128; ++L) {
+      const int row = (L & 7) + 16 * (L >> 4), half = (L >> 3) & 1;
+      for (int kb = 0; kb < 4; ++kb) {
+        // canonical bytes: 2 windows per byte; k-block kb covers windows 8kb..8kb+7 = bytes 4kb..4kb+3
+        const uint8_t* lo = &m->tc_meta[(tm * kTileM + row) * meta_ld + tk * (kTileK / 8) + 4 * kb + 2 * half];
+        const uint8_t* hi = &m->tc_meta[(tm * kTileM + row + 8) * meta_ld + tk * (kTileK / 8) + 4 * kb + 2 * half];
+        meta[L * 4 + kb] = static_cast<uint32_t>(lo[0]) | static_cast<uint32_t>(lo[1]) << 8 |
+                           static_cast<uint32_t>(hi[0]) << 16 | static_cast<uint32_t>(hi[1]) << 24;
+      }
+    }
+    uint32_t* info = reinterpret_cast<uint32_t*>(blk + kInfoOff);
+    info[0] = tc.pdd_len;
+    info[1] = tc.res_cnt;
+    // Chain slot w * 32 + l holds the w-th longest of the four chains of bank l (ties: lower u
+    // first).  Decode thread j takes slot j (rotated by 32 from tile to tile), so the lanes of a
+    // warp sit in 32 different banks and get chains of similar length.
+    uint32_t* hdrs = reinterpret_cast<uint32_t*>(blk + kHdrOff);
+    int chain_at[kChains];
+    for (int bank = 0; bank < 32; ++bank) {
+      int cs[4] = {4 * bank, 4 * bank + 1, 4 * bank + 2, 4 * bank + 3};
+      std::stable_sort(cs, cs + 4, [&](int a, int b) { return tc.len[a] > tc.len[b]; });
+      for (int w = 0; w < 4; ++w) chain_at[w * 32 + bank] = cs[w];
+    }
+    uint8_t* code = blk + kPddOff;
+    for (int j = 0; j < kChains; ++j) {
+      const int c = chain_at[j];
+      hdrs[j] = tc.hdr[c];
+      blk[kLenOff + j] = tc.len[c];
+      if (tc.len[c]) std::memcpy(code, tc.code.data() + tc.code_off[c], tc.len[c]);
+      code += tc.len[c];
+    }
+    if (tc.res_cnt) std::memcpy(blk + kPddOff + align_up(tc.pdd_len, 4), tc.res.data(), 4 * static_cast<size_t>(tc.res_cnt));
+  });
 }
 
 }  // namespace tl3

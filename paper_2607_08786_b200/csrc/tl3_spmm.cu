@@ -228,9 +228,12 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// byte offset of value slot `pos` (row = pos / 64, slot = pos % 64) inside a 128 x 128-byte
-// K-major tile with the 128-byte swizzle: 16-byte chunk index ^= row & 7
-__device__ __forceinline__ uint32_t swizzled_offset(uint32_t pos) { return (pos << 1) ^ ((pos >> 2) & 0x70u); }
+// Positions in a block are bank-major slot coordinates u = bank << 8 | slot-in-window << 7 | row,
+// where bank is the 32-bit word of the 128-byte (swizzled) row that holds the slot's window.  The
+// byte offset of slot u inside the 128 x 128-byte K-major image is therefore a bit-field move:
+// row * 128 + bank * 4 + slot-in-window * 2.  The packer orders both PDD streams by u and gives
+// lane l of a decode warp a chain whose empty slots all lie in bank l.
+__device__ __forceinline__ uint32_t swizzled_offset(uint32_t u) { return ((u & 0x7Fu) << 7) | ((u >> 6) & 0x7Eu); }
 
 template <int NPAD> struct TmemLd;
 template <> struct TmemLd<16> {
@@ -279,8 +282,8 @@ __device__ __forceinline__ void sts_zero16B(uint32_t addr) {
 }
 
 // Algorithm 1 for one chain, one code word (four delta bytes) at a time.  `pos` carries offset_t in its low and
-// offset_r in its high 16 bits, so one add advances both cursors and one shift/xor pair forms both
-// swizzled byte offsets.  Within a round all positions are formed first, then all W_t loads are
+// offset_r in its high 16 bits (both as bank-major coordinates u), so one add advances both cursors
+// and two shift/mask pairs form both byte offsets.  Within a round all positions are formed first, then all W_t loads are
 // issued, then all stores, so that the shared-memory round trips of different entries overlap; the
 // next code word is fetched before the current one is processed.  (Longer rounds measured slower:
 // lanes whose chain has ended only execute predicated-off instructions.)
@@ -290,7 +293,7 @@ __device__ __forceinline__ void sts_zero16B(uint32_t addr) {
 constexpr int kBatch = TL3_DECODE_BATCH;                  // 1, 2 or 4 delta bytes per round of loads and stores
 
 // packed byte offsets (W_t offset low, W_r offset high) of the packed positions `pos`
-__device__ __forceinline__ uint32_t swizzled_offset2(uint32_t pos) { return (pos << 1) ^ ((pos >> 2) & 0x00700070u); }
+__device__ __forceinline__ uint32_t swizzled_offset2(uint32_t pos) { return ((pos & 0x007F007Fu) << 7) | ((pos >> 6) & 0x007E007Eu); }
 
 // Positions are checked (< 8192 slots per tile) before they become addresses; a violation is
 // reported in *bad and the entry is skipped.
@@ -663,9 +666,21 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       const long long seg_end = row_tile_end < t_end ? row_tile_end : t_end;
       const bool complete = (t == row_tile_begin) && (seg_end == row_tile_end);
       const int b = seg & 1;
+      const int c_first = owner_of(row_tile_begin, T, G), c_last = owner_of(row_tile_end - 1, T, G);
+      // A row-tile shared with other CTAs: look at its arrival counter before waiting for the
+      // accumulator.  If every other contributor has arrived by then, this CTA is the last one: it
+      // adds the others' partial sums to its own registers and writes Y directly, without the
+      // partial-sum store, fence and atomic on its way out (the usual case for the segment a CTA
+      // ends with, since the CTAs it shares that row-tile with finished their part earlier).
+      if (!complete && et == 0) {
+        unsigned int seen;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.counters + mt) : "memory");
+        *last_flag = seen == static_cast<unsigned int>(c_last - c_first) ? 2u : 0u;
+      }
       if (!named_bar_all(1 + kGroups, 128, mbar_wait(bar_accfull + 8 * b, (seg >> 1) & 1, wctx, kStEpilogueAccFull))) break;
       TL3_TACC(1)
       tc_fence_after();
+      const bool all_others_in = !complete && *last_flag == 2u;
       constexpr int CH = NPAD < 32 ? NPAD : 32;                 // columns handled per round (register budget)
       const int row = mt * kTileM + et;
       __half* y = a.Y + static_cast<long long>(row) * a.ldy;
@@ -694,6 +709,54 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       // partial sums of a shared row-tile: slot 2*cta + (this row-tile is not the first one of my range)
       const int slot = 2 * blockIdx.x + (t_begin < row_tile_begin ? 1 : 0);
       float* mine = a.partials + static_cast<size_t>(slot) * NPAD * 128 + et;
+      if (all_others_in) {
+        __threadfence();                                          // the others' partial sums, after the counter
+#pragma unroll 1
+        for (int c0 = 0; c0 < NPAD; c0 += 16) {                   // 16 columns at a time (register budget)
+          uint32_t v[CH];                                         // (only the first 16 are used)
+          TmemLd<16>::ld(acc_tmem + c0, v);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          float acc[16];
+#pragma unroll
+          for (int c = 0; c < 16; ++c) acc[c] = 0.f;
+          for (int c_id = c_first; c_id <= c_last; ++c_id) {      // same fixed order as the reduction below
+            if (c_id == static_cast<int>(blockIdx.x)) {
+#pragma unroll
+              for (int c = 0; c < 16; ++c) acc[c] += __uint_as_float(v[c]);
+            } else {
+              const int sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
+              const float* p = a.partials + static_cast<size_t>(sl) * NPAD * 128 + et;
+#pragma unroll
+              for (int c = 0; c < 16; ++c) acc[c] += __ldcg(p + (c0 + c) * 128);
+            }
+          }
+          if (row < a.M) {
+            if (vec_ok) {
+#pragma unroll
+              for (int c = 0; c < 16; c += 8) {
+                uint4 o;
+                __half2 h0 = __floats2half2_rn(acc[c + 0], acc[c + 1]), h1 = __floats2half2_rn(acc[c + 2], acc[c + 3]);
+                __half2 h2 = __floats2half2_rn(acc[c + 4], acc[c + 5]), h3 = __floats2half2_rn(acc[c + 6], acc[c + 7]);
+                o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
+                o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
+                *reinterpret_cast<uint4*>(y + c0 + c) = o;
+              }
+            } else {
+#pragma unroll
+              for (int c = 0; c < 16; ++c)
+                if (c0 + c < a.N) y[c0 + c] = __float2half_rn(acc[c]);
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar_accempty + 8 * b);
+        if (et == 0) a.counters[mt] = 0;                          // leave the workspace cleared
+        named_bar_sync(1 + kGroups, 128);                         // last_flag is rewritten next segment
+        TL3_TACC(2)
+        ++seg;
+        t = seg_end;
+        continue;
+      }
 #pragma unroll 1
       for (int c0 = 0; c0 < NPAD; c0 += CH) {
         uint32_t v[CH];
@@ -711,7 +774,6 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       if (!complete) {
         __threadfence();
         named_bar_sync(1 + kGroups, 128);
-        const int c_first = owner_of(row_tile_begin, T, G), c_last = owner_of(row_tile_end - 1, T, G);
         if (et == 0) {
           const unsigned int old = atomicAdd(a.counters + mt, 1u);
           const bool last = old == static_cast<unsigned int>(c_last - c_first);

@@ -142,67 +142,120 @@ def test_error_codes(tl3):
     assert L.tl3_strerror(-99) == b"unknown error"
 
 
-def _expected_blob_blocks(c, M_pad, K_pad):
-    """The device layout re-derived in numpy from the oracle's container, tile by tile."""
-    H = 64
+def _image_offset(u):
+    """Byte offset of bank-major slot u = bank << 8 | slot-in-window << 7 | row in the value image."""
+    return ((u & 127) << 7) | ((u >> 6) & 0x7E)
+
+
+def _decode_device_blob(blob, M_pad, K_pad):
+    """Algorithm 1 run in numpy over every tile block of a packed blob, as the kernel runs it:
+    parked values move from W_t[tau] to W_r[rho], Residual entries go to W_r, then both sparse
+    operands are expanded with their metadata.  Returns the dense fp16 bit patterns and checks the
+    structure of each block on the way."""
     tiles_m, tiles_k = M_pad // 128, K_pad // 128
-    vals = c.tc_vals.reshape(M_pad, K_pad // 2)
-    meta = c.tc_meta.reshape(M_pad, K_pad // 8)
-    for tm in range(tiles_m):
-        for tk in range(tiles_k):
-            t = tm * tiles_k + tk
-            pdd_off, pdd_len, res_off, res_cnt = (int(x) for x in c.tile_dir[t])
-            v = vals[tm * 128:(tm + 1) * 128, tk * H:(tk + 1) * H].reshape(128, 8, 8)     # row, chunk, 8 values
-            img = np.zeros((128, 8, 8), dtype=np.uint16)
-            for r in range(128):
-                for j in range(8):
-                    img[r, j ^ (r & 7)] = v[r, j]
-            mt = meta[tm * 128:(tm + 1) * 128, tk * 16:(tk + 1) * 16]                         # 16 bytes per row
-            words = np.zeros((128, 4), dtype=np.uint32)
-            for L in range(128):
-                row, half = (L & 7) + 16 * (L >> 4), (L >> 3) & 1
-                for kb in range(4):
-                    lo = mt[row, 4 * kb + 2 * half: 4 * kb + 2 * half + 2].astype(np.uint32)
-                    hi = mt[row + 8, 4 * kb + 2 * half: 4 * kb + 2 * half + 2].astype(np.uint32)
-                    words[L, kb] = lo[0] | lo[1] << 8 | hi[0] << 16 | hi[1] << 24
-            info = np.array([pdd_len, res_cnt, 0, 0], dtype=np.uint32)
-            hdr = (c.chain_tau0[t * 128:(t + 1) * 128].astype(np.uint32) |
-                   c.chain_rho0[t * 128:(t + 1) * 128].astype(np.uint32) << 16)
-            lens = c.chain_len[t * 128:(t + 1) * 128]
-            # chains longest first, ties by row
-            order = sorted(range(128), key=lambda r: (-int(lens[r]), r))
-            starts = np.concatenate([[0], np.cumsum(lens.astype(np.int64))])
-            codes = c.pdd_bytes[pdd_off:pdd_off + pdd_len]
-            pdd = np.concatenate([codes[starts[r]:starts[r + 1]] for r in order]) if pdd_len else codes
-            hdr, lens = hdr[order], lens[order]
-            pad = (-pdd_len) % 4
-            res = (c.res_rho[res_off:res_off + res_cnt].astype(np.uint32) |
-                   c.res_val[res_off:res_off + res_cnt].astype(np.uint32) << 16)
-            block = b"".join([img.tobytes(), words.tobytes(), info.tobytes(), hdr.tobytes(), lens.tobytes(),
-                              pdd.tobytes(), b"\0" * pad, res.tobytes()])
-            block += b"\0" * ((-len(block)) % 16)
-            yield t, block, pdd_len, res_cnt
-
-
-def test_device_blob_layout(tl3, oracle_mod):
-    """Every tile block of the packed blob against an independent numpy construction."""
-    W = wl.Case(0, "pack", 200, 300, 8, 9, 0.45, "magnitude").make_W()     # ragged, some Residual
-    m = tl3.encode(W)
-    c = oracle_mod.encode(W)
-    blob = m.pack()
-    assert blob.size == m.device_bytes() and blob.size % 256 == 0
-    st = m.stats()
-    n_tiles = st["n_tiles"]
+    n_tiles = tiles_m * tiles_k
     directory = blob[256:256 + 16 * n_tiles].view(np.uint32).reshape(n_tiles, 4)
-    seen_end = 0
-    for t, block, pdd_len, res_cnt in _expected_blob_blocks(c, st["M_pad"], st["K_pad"]):
-        off16, nbytes, d_pdd, d_res = (int(x) for x in directory[t])
-        assert (off16 * 16) % 128 == 0 and nbytes % 16 == 0
-        assert (nbytes, d_pdd, d_res) == (len(block), pdd_len, res_cnt)
-        assert off16 * 16 >= seen_end                                   # blocks do not overlap
+    W = np.zeros((M_pad, K_pad), dtype=np.uint16)
+    seen_end = 256 + 16 * n_tiles
+    for t in range(n_tiles):
+        tm, tk = divmod(t, tiles_k)
+        off16, nbytes, pdd_len, res_cnt = (int(x) for x in directory[t])
+        assert (off16 * 16) % 128 == 0 and off16 * 16 >= seen_end             # aligned, no overlap
+        assert nbytes == (19088 + (pdd_len + 3) // 4 * 4 + 4 * res_cnt + 15) // 16 * 16
         seen_end = off16 * 16 + nbytes
-        assert blob[off16 * 16: off16 * 16 + nbytes].tobytes() == block, f"tile {t}"
+        blk = blob[off16 * 16: off16 * 16 + nbytes]
+        img = blk[:16384].view(np.uint16).copy()                              # W_t image, halfword = byte offset / 2
+        meta = blk[16384:18432].view(np.uint32).reshape(128, 4)
+        info = blk[18432:18448].view(np.uint32)
+        assert (int(info[0]), int(info[1])) == (pdd_len, res_cnt)
+        hdr = blk[18448:18960].view(np.uint32)
+        lens = blk[18960:19088]
+        codes = blk[19088:19088 + pdd_len]
+        assert int(lens.astype(np.int64).sum()) == pdd_len
+        res = blk[19088 + (pdd_len + 3) // 4 * 4:][:4 * res_cnt].view(np.uint32)
+        wr = np.zeros(8192, dtype=np.uint16)                                   # W_r image
+        at = 0
+        for j in range(128):
+            n, h = int(lens[j]), int(hdr[j])
+            if j >= 32:
+                assert int(lens[j - 32]) >= n                                  # longest first within a bank
+            if h == 0xFFFFFFFF:
+                assert n == 0
+                continue
+            pt, pr = h & 0xFFFF, h >> 16
+            assert pt < 8192 and pr < 8192 and (pt >> 8) == (j & 31)           # slot j: a chain of bank j % 32
+            chain = pt >> 6
+
+            def move(pt, pr):
+                assert (pt >> 6) == chain                                      # a chain stays in its 64 positions
+                v = img[_image_offset(pt) // 2]
+                assert v & 0x7FFF and wr[_image_offset(pr) // 2] == 0
+                img[_image_offset(pt) // 2] = 0
+                wr[_image_offset(pr) // 2] = v
+
+            move(pt, pr)
+            for b in codes[at:at + n]:
+                dt, dr = int(b) & 15, int(b) >> 4
+                assert dt or dr
+                pt += dt
+                pr += dr
+                if dt and dr:
+                    move(pt, pr)
+            at += n
+        for e in res:
+            u, v = int(e) & 0xFFFF, int(e) >> 16
+            assert u < 8192 and wr[_image_offset(u) // 2] == 0
+            wr[_image_offset(u) // 2] = v
+        nib = np.zeros((128, 32), dtype=np.uint8)                              # metadata nibble of (row, window)
+        for lane in range(128):
+            row, half = (lane & 7) + 16 * (lane >> 4), (lane >> 3) & 1
+            for kb in range(4):
+                w = int(meta[lane, kb])
+                for i in range(4):
+                    nib[row, 8 * kb + 4 * half + i] = (w >> (4 * i)) & 15
+                    nib[row + 8, 8 * kb + 4 * half + i] = (w >> (16 + 4 * i)) & 15
+        for r in range(128):
+            for q in range(32):
+                base = r * 128 + (((q >> 2) ^ (r & 7)) << 4) + (q & 3) * 4    # 128-byte swizzle
+                idx = (int(nib[r, q]) & 3, int(nib[r, q]) >> 2)
+                assert idx[0] < idx[1]
+                for s in range(2):
+                    v = img[(base + 2 * s) // 2]
+                    if v & 0x7FFF:
+                        W[tm * 128 + r, tk * 128 + 4 * q + idx[s]] = v
+                    v = wr[(base + 2 * s) // 2]
+                    if v & 0x7FFF:
+                        assert W[tm * 128 + r, tk * 128 + 4 * q + 2 + s] == 0
+                        W[tm * 128 + r, tk * 128 + 4 * q + 2 + s] = v
     assert seen_end <= blob.size
+    return W
+
+
+@pytest.mark.parametrize("shape,sparsity,mask", [((200, 300), 0.45, "magnitude"), ((256, 384), 0.5, "bernoulli"),
+                                                 ((256, 256), 0.7, "magnitude"), ((128, 256), 0.3, "magnitude"),
+                                                 ((128, 128), 1.0, "bernoulli"), ((128, 128), 0.0, "bernoulli")])
+def test_device_blob_decodes_to_the_matrix(tl3, shape, sparsity, mask):
+    """The packed device image (bank-major re-pairing of the Slot-Filling layer) holds the same
+    matrix: an independent numpy decoder of the blob reproduces W bit for bit, every chain lies in
+    the bank of its lane, chains are longest first, and the blob is hardly larger than the
+    canonical container."""
+    M, K = shape
+    W = wl.Case(0, "pack", M, K, 8, 9, sparsity, mask).make_W()
+    m = tl3.encode(W)
+    blob = m.pack()
+    st = m.stats()
+    assert blob.size == m.device_bytes() and blob.size % 256 == 0
+    ref = np.zeros((st["M_pad"], st["K_pad"]), dtype=np.uint16)
+    ref[:M, :K] = W.view(np.uint16)
+    ref[ref == 0x8000] = 0
+    assert np.array_equal(_decode_device_blob(blob, st["M_pad"], st["K_pad"]), ref)
+
+
+def test_device_blob_size_stays_close_to_canonical(tl3):
+    for sparsity in (0.4, 0.5, 0.6, 0.7):
+        m = tl3.encode(wl.Case(0, "pack", 512, 1024, 8, 9, sparsity, "magnitude").make_W())
+        st = m.stats()
+        assert st["device_bytes"] <= 1.02 * st["canonical_bytes"] + 4096
 
 
 def test_two_rank_plumbing_on_cpu():
