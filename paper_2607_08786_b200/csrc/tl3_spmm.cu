@@ -75,7 +75,7 @@ constexpr uint32_t kTryWaitHintNs = TL3_TRYWAIT_HINT_NS;     // how long one bar
 // status codes written to the workspace status word (0 = ok)
 enum : uint32_t {
   kStProducer = 1, kStDecodeFull = 2, kStDecodeWrFree = 3, kStMmaDecoded = 4, kStMmaAccEmpty = 5,
-  kStEpilogueAccFull = 6, kStDrain = 7, kStClearWrFree = 8, kStDecodeWrReady = 9,
+  kStEpilogueAccFull = 6, kStDrain = 7, kStClearWrFree = 8, kStDecodeWrReady = 9, kStEpilogueTail = 10,
   kStBadBlock = 16           // a block's lengths or a decoded position were out of range (+ detail in bits 8..)
 };
 
@@ -168,6 +168,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
   }
 }
 
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -366,6 +367,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 32);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 33);
   volatile unsigned int* last_flag = reinterpret_cast<volatile unsigned int*>(bars + 34);
+  const uint32_t bar_tail = smem_u32(bars + 36);               // partial sums fetched into the idle stages at the very end
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const long long T = a.total_tiles, G = gridDim.x;
@@ -389,6 +391,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       mbar_init(bar_accempty + 8 * b, 128);
     }
     for (int w = 0; w < kMaxWrBuffers; ++w) { mbar_init(bar_wrready + 8 * w, 64); mbar_init(bar_wrfree + 8 * w, 1); }
+    mbar_init(bar_tail, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -783,21 +786,47 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         named_bar_sync(1 + kGroups, 128);
         if (*last_flag) {
           __threadfence();
-#pragma unroll 1
-          for (int c0 = 0; c0 < NPAD; c0 += CH) {
-            float acc[CH];
-#pragma unroll
-            for (int c = 0; c < CH; ++c) acc[c] = 0.f;
-            for (int c_id = c_first; c_id <= c_last; ++c_id) {    // fixed order: deterministic sum
-              const int sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
-              const float* p = a.partials + static_cast<size_t>(sl) * NPAD * 128 + et;
-#pragma unroll
-              for (int c = 0; c < CH; ++c) acc[c] += __ldcg(p + (c0 + c) * 128);
+          // The last segment of a CTA ends after all of its tiles: the stages are idle then, so the
+          // contributors' partial sums are fetched with one bulk copy each, all in flight at once,
+          // instead of one round trip of loads per contributor.
+          constexpr uint32_t kSlotBytes = NPAD * 128u * 4u;
+          const int n_contrib = c_last - c_first + 1;
+          const bool staged = seg_end == t_end && static_cast<uint32_t>(n_contrib) * kSlotBytes <= static_cast<uint32_t>(S) * a.stage_stride;
+          bool fetched = true;
+          if (staged) {
+            if (et == 0) {
+              fence_proxy_async_all();
+              mbar_arrive_expect_tx(bar_tail, static_cast<uint32_t>(n_contrib) * kSlotBytes);
+              for (int c_id = c_first, k = 0; c_id <= c_last; ++c_id, ++k) {
+                const int sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
+                bulk_copy_g2s(smem_base + static_cast<uint32_t>(k) * kSlotBytes, a.partials + static_cast<size_t>(sl) * NPAD * 128, kSlotBytes, bar_tail);
+              }
             }
-            uint32_t v[CH];
+            fetched = mbar_wait(bar_tail, 0, wctx, kStEpilogueTail);
+          }
+          if (fetched) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < NPAD; c0 += CH) {
+              float acc[CH];
 #pragma unroll
-            for (int c = 0; c < CH; ++c) v[c] = __float_as_uint(acc[c]);
-            store_y(v, c0);
+              for (int c = 0; c < CH; ++c) acc[c] = 0.f;
+              for (int c_id = c_first, k = 0; c_id <= c_last; ++c_id, ++k) {    // fixed order: deterministic sum
+                if (staged) {
+                  const uint32_t p = smem_base + (static_cast<uint32_t>(k) * NPAD * 128u + static_cast<uint32_t>(et)) * 4u;
+#pragma unroll
+                  for (int c = 0; c < CH; ++c) acc[c] += __uint_as_float(lds_u32(p + static_cast<uint32_t>(c0 + c) * 512u));
+                } else {
+                  const int sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
+                  const float* p = a.partials + static_cast<size_t>(sl) * NPAD * 128 + et;
+#pragma unroll
+                  for (int c = 0; c < CH; ++c) acc[c] += __ldcg(p + (c0 + c) * 128);
+                }
+              }
+              uint32_t v[CH];
+#pragma unroll
+              for (int c = 0; c < CH; ++c) v[c] = __float_as_uint(acc[c]);
+              store_y(v, c0);
+            }
           }
         }
         named_bar_sync(1 + kGroups, 128);                         // last_flag may be rewritten next segment
