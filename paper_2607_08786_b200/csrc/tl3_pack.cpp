@@ -8,7 +8,8 @@
 // banks.  Here both streams are ordered bank-major -- a slot's coordinate is
 //     u = bank << 8 | slot-in-window << 7 | row,      bank = word of the 128-byte swizzled row
 // -- the i-th surplus element in that order is parked in the i-th selected empty slot in that
-// order, and chain c holds the pairs whose empty slot has u >> 6 == c.  Lane l of a decode warp
+// order, and the pairs whose empty slot lies in bank b are cut into four chains of equal count.
+// Lane l of a decode warp
 // takes a chain of bank l, so its loads and stores in W_t never collide with another lane's, and
 // its stores in W_r land in bank l or a neighbour.  It is the same format (Sec. 3.2: values parked
 // in empty slots, 16-bit absolute starts, 4-bit delta pairs, dummy points, Residual list) over a
@@ -47,7 +48,7 @@ static inline uint32_t image_offset(uint32_t u) { return ((u & 127u) << 7) | ((u
 namespace {
 
 constexpr int kSlots = kTileM * kH;      // 8192
-constexpr int kChains = 128;             // u >> 6
+constexpr int kChains = 128;             // four per bank
 
 struct TileCode {
   uint32_t pdd_len = 0, res_cnt = 0;
@@ -93,42 +94,69 @@ void build_tile(const tl3_matrix* m, int64_t tm, int64_t tk, TileCode& tc) {
     }
     byte_at += len;
   }
-  // empty slots in u order (every slot whose value is zero: kept values are non-zero), per chain
-  uint32_t cand_count[kChains];
+  // Empty slots in u order (every slot whose value is zero: kept values are non-zero), counted per
+  // bank.  n_pairs <= their number (the canonical encoder parked each element in an empty slot).
+  // Bank b gets a share of the parked elements proportional to its empty slots; its empty slots
+  // are cut into four runs of equal count, and run q uses its first quota(b)/4 slots.  So the
+  // parked elements spread evenly over the tile however many empty slots stay unused, every
+  // chain is a dense run of empty slots (small deltas), and the four chains of a bank are equally
+  // long.
+  uint32_t cand_in_bank[32];
   uint32_t n_cand = 0;
-  static thread_local std::vector<uint8_t> cand(kSlots);
-  for (int c = 0; c < kChains; ++c) {
+  static thread_local std::vector<uint16_t> cand;         // empty slots, in u order
+  cand.clear();
+  for (int b = 0; b < 32; ++b) {
     uint32_t n = 0;
-    for (uint32_t u = 64u * c; u < 64u * c + 64u; ++u) {
-      const bool e = (tc.vals[pos_of_u(u)] & 0x7FFFu) == 0;
-      cand[u] = e;
-      n += e;
-    }
-    cand_count[c] = n;
+    for (uint32_t u = 256u * b; u < 256u * b + 256u; ++u)
+      if ((tc.vals[pos_of_u(u)] & 0x7FFFu) == 0) { cand.push_back(static_cast<uint16_t>(u)); ++n; }
+    cand_in_bank[b] = n;
     n_cand += n;
   }
-  // n_pairs <= n_cand (the canonical encoder parked each element in an empty slot).  Chain c
-  // uses the first quota(c) of its empty slots, quotas proportional to what the chain has, so
-  // the parked elements spread evenly over chains however many empty slots stay unused.
+  n_pairs = 0;
+  for (int u = 0; u < kSlots; ++u) n_pairs += sflag[u];
+  static thread_local std::vector<uint16_t> sel;          // selected empty slots, in u order
+  sel.clear();
+  uint32_t sel_in_chain[kChains];
+  {
+    uint64_t cum = 0;
+    size_t base = 0;                      // first candidate of the bank
+    uint32_t carry = 0;
+    for (int b = 0; b < 32; ++b) {
+      const uint64_t lo = n_cand ? cum * n_pairs / n_cand : 0;
+      cum += cand_in_bank[b];
+      const uint64_t hi = n_cand ? cum * n_pairs / n_cand : 0;
+      const uint32_t n_b = static_cast<uint32_t>(hi - lo), N_b = cand_in_bank[b];
+      for (uint32_t q = 0; q < 4; ++q) {
+        const uint32_t first = N_b * q / 4, size = N_b * (q + 1) / 4 - first;
+        const uint32_t want = n_b * (q + 1) / 4 - n_b * q / 4 + carry;
+        const uint32_t take = want < size ? want : size;
+        carry = want - take;
+        for (uint32_t i = 0; i < take; ++i) sel.push_back(cand[base + first + i]);
+        sel_in_chain[4 * b + q] = take;
+      }
+      base += N_b;
+    }
+  }
+  // Chains: one per run, so the four warps of a decode group finish a tile at about the same time.
   tc.code.clear();
   tc.res.clear();
   uint32_t ur = 0;                        // cursor in the surplus stream
-  auto next_surplus = [&]() { while (!sflag[ur]) ++ur; return ur++; };
-  uint64_t cum = 0;
+  auto next_surplus = [&]() {
+    while (ur < static_cast<uint32_t>(kSlots) && !sflag[ur]) ++ur;
+    return ur < static_cast<uint32_t>(kSlots) ? ur++ : 0xFFFFFFFFu;
+  };
+  size_t at = 0;                          // cursor in sel
   for (int c = 0; c < kChains; ++c) {
-    const uint64_t lo = n_cand ? cum * n_pairs / n_cand : 0;
-    cum += cand_count[c];
-    const uint64_t hi = n_cand ? cum * n_pairs / n_cand : 0;
-    uint32_t quota = static_cast<uint32_t>(hi - lo);
+    const uint32_t count = sel_in_chain[c];
     tc.hdr[c] = 0xFFFFFFFFu;
     tc.len[c] = 0;
     tc.code_off[c] = static_cast<uint32_t>(tc.code.size());
     uint32_t prev_t = 0, prev_r = 0, n_bytes = 0;
     bool first = true, overflow = false;
-    for (uint32_t u = 64u * c; quota && u < 64u * c + 64u; ++u) {
-      if (!cand[u]) continue;
-      --quota;
+    for (uint32_t i = 0; i < count; ++i) {
+      const uint32_t u = sel[at++];
       const uint32_t r_u = next_surplus();
+      if (r_u == 0xFFFFFFFFu) break;
       const uint16_t v = sval[r_u];
       if (overflow) { tc.res.push_back(r_u | static_cast<uint32_t>(v) << 16); continue; }
       if (first) {

@@ -184,10 +184,10 @@ def _decode_device_blob(blob, M_pad, K_pad):
                 continue
             pt, pr = h & 0xFFFF, h >> 16
             assert pt < 8192 and pr < 8192 and (pt >> 8) == (j & 31)           # slot j: a chain of bank j % 32
-            chain = pt >> 6
+            bank = pt >> 8
 
             def move(pt, pr):
-                assert (pt >> 6) == chain                                      # a chain stays in its 64 positions
+                assert (pt >> 8) == bank                                       # a chain stays in the bank of its lane
                 v = img[_image_offset(pt) // 2]
                 assert v & 0x7FFF and wr[_image_offset(pr) // 2] == 0
                 img[_image_offset(pt) // 2] = 0
