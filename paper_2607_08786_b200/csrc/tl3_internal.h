@@ -53,12 +53,13 @@ namespace tl3 {
 //   +18448  chain starts u32[128]: tau0 | rho0 << 16 (0xFFFFFFFF = empty chain) in the bank-major
 //           slot coordinate u = bank << 8 | slot-in-window << 7 | row; chain slot w * 32 + l holds
 //           the w-th longest of the four chains whose empty slots lie in bank l
-//   +18960  chain lengths u8[128], same order
-//   +19088  PDD delta bytes, chain after chain in that order, padded to 4 bytes
+//   +18960  u16[129]: byte offset of each chain's code within the PDD area, same order, and the
+//           total as the last entry (a chain's length is the difference to the next offset)
+//   +19224  PDD delta bytes, chain after chain in that order, padded to 4 bytes
 //   +...    Residual entries u32[res_cnt]: u of the element | value << 16, padded to 16 bytes
 constexpr int kTileM = 128, kTileK = 128, kH = 64;
 constexpr uint32_t kValsBytes = 16384, kMetaOff = 16384, kMetaBytes = 2048;
-constexpr uint32_t kInfoOff = 18432, kHdrOff = 18448, kLenOff = 18960, kPddOff = 19088;
+constexpr uint32_t kInfoOff = 18432, kHdrOff = 18448, kLenOff = 18960, kPddOff = 19224;
 constexpr uint32_t kBlockAlign = 128;
 
 struct DirEntry {

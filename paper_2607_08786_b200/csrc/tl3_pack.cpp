@@ -291,10 +291,11 @@ void pack_device_blob(const tl3_matrix* m, uint8_t* out) {
     for (int j = 0; j < kChains; ++j) {
       const int c = chain_at[j];
       hdrs[j] = tc.hdr[c];
-      blk[kLenOff + j] = tc.len[c];
+      reinterpret_cast<uint16_t*>(blk + kLenOff)[j] = static_cast<uint16_t>(code - (blk + kPddOff));
       if (tc.len[c]) std::memcpy(code, tc.code.data() + tc.code_off[c], tc.len[c]);
       code += tc.len[c];
     }
+    reinterpret_cast<uint16_t*>(blk + kLenOff)[kChains] = static_cast<uint16_t>(code - (blk + kPddOff));
     if (tc.res_cnt) std::memcpy(blk + kPddOff + align_up(tc.pdd_len, 4), tc.res.data(), 4 * static_cast<size_t>(tc.res_cnt));
   });
 }

@@ -8,8 +8,8 @@
 //     of shared-memory stages (Sec. 4.2 "Efficient Matrix Loading": W streamed tile by tile, X
 //     small enough to live in L2);
 //   * four groups of four decode warps take the tiles in turn: copy the 2-bit metadata to tensor
-//     memory, run Algorithm 1 (one PDD chain per thread; chain byte offsets by a warp-shuffle
-//     prefix sum of the chain lengths) moving each parked value from W_t to a second 2:4 operand
+//     memory, run Algorithm 1 (one PDD chain per thread, lane l on a chain whose empty slots lie
+//     in shared-memory bank l) moving each parked value from W_t to a second 2:4 operand
 //     W_r and zeroing its slot, and scatter the Residual entries into W_r as well
 //     (Sec. 4.3; surplus weights always sit at in-window index 2 or 3, so W_r's metadata is the
 //     constant pattern {2,3}); two more warps clear each W_r buffer as soon as its MMAs are done;
@@ -591,11 +591,18 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       ok = ok && mbar_wait(bar_full + 8 * s, ph, wctx, kStDecodeFull);
       TL3_TACC(2)
       const uint32_t stage = smem_base + static_cast<uint32_t>(s) * a.stage_stride;
-      uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0, quad = 0, hdr = 0xFFFFFFFFu;
+      uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0, span = 0, hdr = 0xFFFFFFFFu, pdd_len = 0, res_cnt = 0;
       if (ok) {
         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(m0), "=r"(m1), "=r"(m2), "=r"(m3) : "r"(stage + kMetaOff + r * 16));
-        quad = lds_u32(stage + kLenOff + lane * 4);
+        {
+          uint16_t o0, o1;
+          asm volatile("ld.shared.u16 %0, [%1];" : "=h"(o0) : "r"(stage + kLenOff + cr * 2));
+          asm volatile("ld.shared.u16 %0, [%1];" : "=h"(o1) : "r"(stage + kLenOff + cr * 2 + 2));
+          span = static_cast<uint32_t>(o0) | static_cast<uint32_t>(o1) << 16;
+        }
         hdr = lds_u32(stage + kHdrOff + cr * 4);
+        pdd_len = lds_u32(stage + kInfoOff);
+        res_cnt = lds_u32(stage + kInfoOff + 4);
       }
       if (!__all_sync(0xFFFFFFFFu, ok)) break;
       if (r == 0) TL3_STAMP(i, 2)
@@ -604,29 +611,13 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
                      ::"r"(tmem_base + lane_base + kColMetaT + 4 * wb), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
       }
-      // byte offset of this thread's chain = exclusive prefix sum of the chain lengths.
-      // Each warp scans all 128 lengths (4 per lane) with shuffles; no cross-warp exchange.
-      uint32_t off, len;
-      {
-        const uint32_t qsum = __dp4a(quad, 0x01010101u, 0u);
-        uint32_t incl = qsum;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-          const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-          if (lane >= d) incl += n;
-        }
-        const int src = cr >> 2;                                 // lane that holds my chain's quad
-        const uint32_t q = __shfl_sync(0xFFFFFFFFu, quad, src);
-        const uint32_t excl = __shfl_sync(0xFFFFFFFFu, incl - qsum, src);
-        const int sub = cr & 3;
-        off = excl + __dp4a(q & ((1u << (8 * sub)) - 1u), 0x01010101u, 0u);
-        len = (q >> (8 * sub)) & 0xFFu;
-      }
+      // byte offset and length of this thread's chain: the block lists where each chain's code starts
+      const uint32_t off = span & 0xFFFFu, len = (span >> 16) - off;
       TL3_TACC(4)
       uint32_t bad = 0;
-      const uint32_t pdd_len = lds_u32(stage + kInfoOff), res_cnt = lds_u32(stage + kInfoOff + 4);
       const uint32_t room = a.x_offset - kPddOff;               // bytes a block may use after its fixed part
-      const bool lens_ok = pdd_len <= room && res_cnt <= room / 4 && ((pdd_len + 3u) & ~3u) + 4u * res_cnt <= room && off + len <= pdd_len;
+      const bool lens_ok = pdd_len <= room && res_cnt <= room / 4 && ((pdd_len + 3u) & ~3u) + 4u * res_cnt <= room &&
+                           (span >> 16) >= off && len <= 255u && off + len <= pdd_len;
       if (lens_ok) decode_chain(stage, wr, hdr, stage + kPddOff + off, len, &bad);
       else bad = 3u;
       __syncwarp();

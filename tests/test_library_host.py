@@ -161,7 +161,7 @@ def _decode_device_blob(blob, M_pad, K_pad):
         tm, tk = divmod(t, tiles_k)
         off16, nbytes, pdd_len, res_cnt = (int(x) for x in directory[t])
         assert (off16 * 16) % 128 == 0 and off16 * 16 >= seen_end             # aligned, no overlap
-        assert nbytes == (19088 + (pdd_len + 3) // 4 * 4 + 4 * res_cnt + 15) // 16 * 16
+        assert nbytes == (19224 + (pdd_len + 3) // 4 * 4 + 4 * res_cnt + 15) // 16 * 16
         seen_end = off16 * 16 + nbytes
         blk = blob[off16 * 16: off16 * 16 + nbytes]
         img = blk[:16384].view(np.uint16).copy()                              # W_t image, halfword = byte offset / 2
@@ -169,16 +169,18 @@ def _decode_device_blob(blob, M_pad, K_pad):
         info = blk[18432:18448].view(np.uint32)
         assert (int(info[0]), int(info[1])) == (pdd_len, res_cnt)
         hdr = blk[18448:18960].view(np.uint32)
-        lens = blk[18960:19088]
-        codes = blk[19088:19088 + pdd_len]
-        assert int(lens.astype(np.int64).sum()) == pdd_len
-        res = blk[19088 + (pdd_len + 3) // 4 * 4:][:4 * res_cnt].view(np.uint32)
+        offs = blk[18960:18960 + 2 * 129].view(np.uint16).astype(np.int64)       # where each chain's code starts
+        assert offs[0] == 0 and offs[128] == pdd_len and (np.diff(offs) >= 0).all() and (np.diff(offs) <= 255).all()
+        lens = np.diff(offs)
+        codes = blk[19224:19224 + pdd_len]
+        res = blk[19224 + (pdd_len + 3) // 4 * 4:][:4 * res_cnt].view(np.uint32)
         wr = np.zeros(8192, dtype=np.uint16)                                   # W_r image
         at = 0
         for j in range(128):
             n, h = int(lens[j]), int(hdr[j])
             if j >= 32:
                 assert int(lens[j - 32]) >= n                                  # longest first within a bank
+            assert at == offs[j]
             if h == 0xFFFFFFFF:
                 assert n == 0
                 continue
