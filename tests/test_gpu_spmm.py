@@ -136,6 +136,15 @@ def test_degenerate_matrices(tl3, oracle_mod):
     check(oracle_mod, T, X, Y)
 
 
+def test_device_chain_overflow(tl3, oracle_mod):
+    """A tile whose device-image chains overflow into the Residual list (see special_cases)."""
+    from special_cases import clustered_surplus_tile
+    W = np.tile(clustered_surplus_tile(), (2, 3))
+    X = np.random.default_rng(5).standard_normal((384, 16)).astype(np.float16)
+    Y, _ = run_gpu(tl3, W, X)
+    check(oracle_mod, W, X, Y)
+
+
 def test_fewer_stages_than_decode_groups(tl3, oracle_mod):
     """Large blocks (heavy Residual layer) and a wide X leave room for only two or three stages in
     shared memory; several tiles per CTA, so the ring wraps many times."""

@@ -170,7 +170,7 @@ def _decode_device_blob(blob, M_pad, K_pad):
         assert (int(info[0]), int(info[1])) == (pdd_len, res_cnt)
         hdr = blk[18448:18960].view(np.uint32)
         offs = blk[18960:18960 + 2 * 129].view(np.uint16).astype(np.int64)       # where each chain's code starts
-        assert offs[0] == 0 and offs[128] == pdd_len and (np.diff(offs) >= 0).all() and (np.diff(offs) <= 255).all()
+        assert offs[0] == 0 and offs[128] == pdd_len and (np.diff(offs) >= 0).all() and (np.diff(offs) <= 12).all()
         lens = np.diff(offs)
         codes = blk[19224:19224 + pdd_len]
         res = blk[19224 + (pdd_len + 3) // 4 * 4:][:4 * res_cnt].view(np.uint32)
@@ -253,11 +253,25 @@ def test_device_blob_decodes_to_the_matrix(tl3, shape, sparsity, mask):
     assert np.array_equal(_decode_device_blob(blob, st["M_pad"], st["K_pad"]), ref)
 
 
+def test_device_chain_overflow_goes_to_the_residual_list(tl3):
+    """A chain of the device image is cut when it is full (here: because two consecutive pairs lie
+    thousands of positions apart); what is cut off travels in the Residual list, and the blob
+    still decodes to the matrix."""
+    from special_cases import clustered_surplus_tile
+    W = clustered_surplus_tile()
+    m = tl3.encode(W)
+    assert m.stats()["n_res"] == 0                                   # nothing in the canonical Residual layer
+    blob = m.pack()
+    directory = blob[256:272].view(np.uint32)
+    assert int(directory[3]) > 0                                       # but the device image has Residual entries
+    assert np.array_equal(_decode_device_blob(blob, 128, 128), W.view(np.uint16))
+
+
 def test_device_blob_size_stays_close_to_canonical(tl3):
     for sparsity in (0.4, 0.5, 0.6, 0.7):
         m = tl3.encode(wl.Case(0, "pack", 512, 1024, 8, 9, sparsity, "magnitude").make_W())
         st = m.stats()
-        assert st["device_bytes"] <= 1.02 * st["canonical_bytes"] + 4096
+        assert st["device_bytes"] <= 1.035 * st["canonical_bytes"] + 4096
 
 
 def test_two_rank_plumbing_on_cpu():
