@@ -49,17 +49,17 @@ namespace tl3 {
 //   +16384  metadata 128 x 16 B: word kb of entry L is the TMEM word of lane L for k-block kb:
 //                    bits 0-15 = nibbles of windows 8kb+4h .. 8kb+4h+3 of row (L&7)+16(L>>4),
 //                    bits 16-31 = the same windows of that row + 8, with h = (L>>3)&1
-//   +18432  u32[4]: pdd_len, res_cnt, 0, 0
+//   +18432  u32[4]: pdd_len, res_cnt, n_words, 0
 //   +18448  chain starts u32[128]: tau0 | rho0 << 16 (0xFFFFFFFF = empty chain) in the bank-major
 //           slot coordinate u = bank << 8 | slot-in-window << 7 | row; chain slot w * 32 + l holds
 //           the w-th longest of the four chains whose empty slots lie in bank l
-//   +18960  u16[129]: byte offset of each chain's code within the PDD area, same order, and the
-//           total as the last entry (a chain's length is the difference to the next offset)
-//   +19224  PDD delta bytes, chain after chain in that order, padded to 4 bytes
+//   +18960  PDD code words, transposed: word k (delta bytes 4k..4k+3) of chain slot j at byte
+//           (k * 128 + j) * 4; every chain of the tile has n_words <= 3 of them, padded with zero
+//           bytes (dummy points); pdd_len = 512 * n_words
 //   +...    Residual entries u32[res_cnt]: u of the element | value << 16, padded to 16 bytes
 constexpr int kTileM = 128, kTileK = 128, kH = 64;
 constexpr uint32_t kValsBytes = 16384, kMetaOff = 16384, kMetaBytes = 2048;
-constexpr uint32_t kInfoOff = 18432, kHdrOff = 18448, kLenOff = 18960, kPddOff = 19224;
+constexpr uint32_t kInfoOff = 18432, kHdrOff = 18448, kPddOff = 18960;
 constexpr uint32_t kBlockAlign = 128;
 
 struct DirEntry {

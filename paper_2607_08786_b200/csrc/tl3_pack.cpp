@@ -15,7 +15,7 @@
 // in empty slots, 16-bit absolute starts, 4-bit delta pairs, dummy points, Residual list) over a
 // different enumeration of the tile's slots.  Kept values, metadata and the canonical Residual
 // elements are carried over as they are; of the canonical parked elements, those that do not fit
-// the first three code words of their chain become Residual entries of the device image.
+// the code words of their chain (at most three) become Residual entries of the device image.
 #include <algorithm>
 #include <atomic>
 #include <cstring>
@@ -50,12 +50,10 @@ namespace {
 
 constexpr int kSlots = kTileM * kH;      // 8192
 constexpr int kChains = 128;             // four per bank
-// A chain is cut after three code words (12 delta bytes); what its run of empty slots holds beyond
-// that (about 8 % of the parked elements at 50 % sparsity) travels as Residual entries, which the
-// decode warps scatter all at once instead of one more serial round of the slowest chains.
-// Measured on 20480 x 5120, N = 16: no cut 32.2 us, 16 bytes 31.4, 14 31.5, 12 30.1, 10 30.9, 8 31.5
-// (the Residual entries cost 4 bytes each: the blob grows from 0.640 to 0.648 of dense at 12).
-constexpr uint32_t kChainCap = 12;
+// (How long a chain may get is decided per tile in build_tile.  Measured on 20480 x 5120, N = 16,
+// with chains of any length 32.2 us, cut after 16 / 14 / 12 / 10 / 8 delta bytes 31.4 / 31.5 /
+// 30.1 / 30.9 / 31.5 us: the MMA of a tile waits for its slowest chain, while Residual entries are
+// scattered by whichever lane is free.)
 
 struct TileCode {
   uint32_t pdd_len = 0, res_cnt = 0;
@@ -144,57 +142,74 @@ void build_tile(const tl3_matrix* m, int64_t tm, int64_t tk, TileCode& tc) {
       base += N_b;
     }
   }
-  // Chains: one per run, so the four warps of a decode group finish a tile at about the same time.
+  // Pairs: the i-th selected empty slot takes the i-th surplus element (both in u order).
+  static thread_local std::vector<uint16_t> sur;          // surplus elements, in u order
+  sur.clear();
+  for (uint32_t u = 0; u < static_cast<uint32_t>(kSlots); ++u)
+    if (sflag[u]) sur.push_back(static_cast<uint16_t>(u));
+  const size_t n_use = sel.size() < sur.size() ? sel.size() : sur.size();
+  // Chains: one per run, so the four warps of a decode group finish a tile at about the same
+  // time.  Every chain of a tile gets the same number of code words, n_words <= 3 (zero bytes pad
+  // the shorter ones); what a run holds beyond 4 * n_words delta bytes travels as Residual
+  // entries.  n_words is the count that makes the block smallest (512 bytes per code word against
+  // 4 bytes per Residual entry): three at 50 % sparsity, one or two where few elements are parked.
+  auto delta_bytes = [](uint32_t gt, uint32_t gr) { return (gt - 1) / 15 + (gr - 1) / 15 + 1; };
+  uint32_t beyond[4] = {0, 0, 0, 0};      // entries whose last delta byte lies beyond 0, 4, 8, 12 bytes
+  {
+    size_t i = 0;
+    for (int c = 0; c < kChains; ++c) {
+      uint32_t end = 0;
+      for (uint32_t k = 0; k < sel_in_chain[c] && i < n_use; ++k, ++i) {
+        if (k == 0) continue;             // the first pair of a chain sits in its header
+        end += delta_bytes(static_cast<uint32_t>(sel[i] - sel[i - 1]), static_cast<uint32_t>(sur[i] - sur[i - 1]));
+        for (int w = 0; w < 4; ++w) beyond[w] += end > 4u * w;
+      }
+    }
+  }
+  uint32_t n_words = 0;
+  for (uint32_t w = 1; w < 4; ++w)
+    if (512u * w + 4u * beyond[w] < 512u * n_words + 4u * beyond[n_words]) n_words = w;
+  const uint32_t cap = 4u * n_words;
   tc.code.clear();
   tc.res.clear();
-  uint32_t ur = 0;                        // cursor in the surplus stream
-  auto next_surplus = [&]() {
-    while (ur < static_cast<uint32_t>(kSlots) && !sflag[ur]) ++ur;
-    return ur < static_cast<uint32_t>(kSlots) ? ur++ : 0xFFFFFFFFu;
-  };
-  size_t at = 0;                          // cursor in sel
-  for (int c = 0; c < kChains; ++c) {
-    const uint32_t count = sel_in_chain[c];
-    tc.hdr[c] = 0xFFFFFFFFu;
-    tc.len[c] = 0;
-    tc.code_off[c] = static_cast<uint32_t>(tc.code.size());
-    uint32_t prev_t = 0, prev_r = 0, n_bytes = 0;
-    bool first = true, overflow = false;
-    for (uint32_t i = 0; i < count; ++i) {
-      const uint32_t u = sel[at++];
-      const uint32_t r_u = next_surplus();
-      if (r_u == 0xFFFFFFFFu) break;
-      const uint16_t v = sval[r_u];
-      if (overflow) { tc.res.push_back(r_u | static_cast<uint32_t>(v) << 16); continue; }
-      if (first) {
-        tc.hdr[c] = u | r_u << 16;
-        first = false;
-      } else {
-        uint32_t gt = u - prev_t, gr = r_u - prev_r;
-        const uint32_t need = (gt - 1) / 15 + (gr - 1) / 15 + 1;
-        if (n_bytes + need > kChainCap) {   // the chain is full: the rest of its run goes to the Residual list
-          overflow = true;
-          tc.res.push_back(r_u | static_cast<uint32_t>(v) << 16);
-          continue;
+  {
+    size_t i = 0;
+    for (int c = 0; c < kChains; ++c) {
+      tc.hdr[c] = 0xFFFFFFFFu;
+      tc.len[c] = 0;
+      tc.code_off[c] = static_cast<uint32_t>(tc.code.size());
+      uint32_t n_bytes = 0;
+      bool cut = false;
+      for (uint32_t k = 0; k < sel_in_chain[c] && i < n_use; ++k, ++i) {
+        const uint32_t u = sel[i], r_u = sur[i];
+        const uint16_t v = sval[r_u];
+        if (k == 0) {
+          tc.hdr[c] = u | r_u << 16;
+        } else {
+          uint32_t gt = u - sel[i - 1], gr = r_u - sur[i - 1];
+          const uint32_t need = delta_bytes(gt, gr);
+          if (cut || n_bytes + need > cap) {            // the chain is full: the rest of its run goes to the Residual list
+            cut = true;
+            tc.res.push_back(r_u | static_cast<uint32_t>(v) << 16);
+            continue;
+          }
+          while (gt > 15) { tc.code.push_back(0x0F); gt -= 15; }     // dummy points (a zero nibble moves nothing)
+          while (gr > 15) { tc.code.push_back(0xF0); gr -= 15; }
+          tc.code.push_back(static_cast<uint8_t>(gt | gr << 4));
+          n_bytes += need;
         }
-        while (gt > 15) { tc.code.push_back(0x0F); gt -= 15; }     // dummy points (a zero nibble moves nothing)
-        while (gr > 15) { tc.code.push_back(0xF0); gr -= 15; }
-        tc.code.push_back(static_cast<uint8_t>(gt | gr << 4));
-        n_bytes += need;
+        tc.vals[pos_of_u(u)] = v;
       }
-      prev_t = u;
-      prev_r = r_u;
-      tc.vals[pos_of_u(u)] = v;
+      tc.len[c] = static_cast<uint8_t>(n_bytes);
     }
-    tc.len[c] = static_cast<uint8_t>(n_bytes);
   }
+  for (size_t i = n_use; i < sur.size(); ++i)               // none left unless the container had more parked elements than empty slots
+    tc.res.push_back(sur[i] | static_cast<uint32_t>(sval[sur[i]]) << 16);
   // canonical Residual entries, in the same coordinate
   const uint32_t res_off = m->tile_dir[t * 4 + 2], res_cnt = m->tile_dir[t * 4 + 3];
   for (uint32_t j = 0; j < res_cnt; ++j)
     tc.res.push_back(u_of_pos(m->res_rho[res_off + j]) | static_cast<uint32_t>(m->res_val[res_off + j]) << 16);
-  for (; ur < static_cast<uint32_t>(kSlots); ++ur)          // none left unless the container had more parked elements than empty slots
-    if (sflag[ur]) tc.res.push_back(ur | static_cast<uint32_t>(sval[ur]) << 16);
-  tc.pdd_len = static_cast<uint32_t>(tc.code.size());
+  tc.pdd_len = n_words * 4u * kChains;                      // every chain takes the same number of code words
   tc.res_cnt = static_cast<uint32_t>(tc.res.size());
 }
 
@@ -294,15 +309,17 @@ void pack_device_blob(const tl3_matrix* m, uint8_t* out) {
       std::stable_sort(cs, cs + 4, [&](int a, int b) { return tc.len[a] > tc.len[b]; });
       for (int w = 0; w < 4; ++w) chain_at[w * 32 + bank] = cs[w];
     }
+    // code words, transposed: word k of chain slot j at byte (k * 128 + j) * 4, every chain padded
+    // with zero bytes (dummy points that move nothing) to the tile's code-word count
+    const uint32_t n_words = tc.pdd_len / (4u * kChains);
     uint8_t* code = blk + kPddOff;
     for (int j = 0; j < kChains; ++j) {
       const int c = chain_at[j];
       hdrs[j] = tc.hdr[c];
-      reinterpret_cast<uint16_t*>(blk + kLenOff)[j] = static_cast<uint16_t>(code - (blk + kPddOff));
-      if (tc.len[c]) std::memcpy(code, tc.code.data() + tc.code_off[c], tc.len[c]);
-      code += tc.len[c];
+      for (uint32_t k = 0; k < tc.len[c]; ++k)
+        code[((k >> 2) * kChains + static_cast<uint32_t>(j)) * 4u + (k & 3u)] = tc.code[tc.code_off[c] + k];
     }
-    reinterpret_cast<uint16_t*>(blk + kLenOff)[kChains] = static_cast<uint16_t>(code - (blk + kPddOff));
+    info[2] = n_words;
     if (tc.res_cnt) std::memcpy(blk + kPddOff + align_up(tc.pdd_len, 4), tc.res.data(), 4 * static_cast<size_t>(tc.res_cnt));
   });
 }

@@ -282,30 +282,28 @@ __device__ __forceinline__ void sts_zero16B(uint32_t addr) {
   asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
 }
 
-// Algorithm 1 for one chain, one code word (four delta bytes) at a time.  `pos` carries offset_t in its low and
-// offset_r in its high 16 bits (both as bank-major coordinates u), so one add advances both cursors
-// and two shift/mask pairs form both byte offsets.  Within a round all positions are formed first, then all W_t loads are
-// issued, then all stores, so that the shared-memory round trips of different entries overlap; the
-// next code word is fetched before the current one is processed.  (Longer rounds measured slower:
-// lanes whose chain has ended only execute predicated-off instructions.)
-#ifndef TL3_DECODE_BATCH
-#define TL3_DECODE_BATCH 4
-#endif
-constexpr int kBatch = TL3_DECODE_BATCH;                  // 1, 2 or 4 delta bytes per round of loads and stores
+// Algorithm 1 for one chain, one code word (four delta bytes) at a time.  `pos` carries offset_t in
+// its low and offset_r in its high 16 bits (both as bank-major coordinates u), so one add advances
+// both cursors and two shift/mask pairs form both byte offsets.  Within a round all positions are
+// formed first, then all W_t loads are issued, then all stores, so that the shared-memory round
+// trips of different entries overlap.  (Rounds of two code words, and a software-pipelined loop
+// that issues the next round's loads before this round's stores, both measured slower.)
 
 // packed byte offsets (W_t offset low, W_r offset high) of the packed positions `pos`
 __device__ __forceinline__ uint32_t swizzled_offset2(uint32_t pos) { return ((pos & 0x007F007Fu) << 7) | ((pos >> 6) & 0x007E007Eu); }
 
 // Positions are checked (< 8192 slots per tile) before they become addresses; a violation is
-// reported in *bad and the entry is skipped.
-__device__ __forceinline__ void decode_chain(uint32_t stage, uint32_t wr, uint32_t hdr, uint32_t code_addr, uint32_t len, uint32_t* bad) {
+// reported in *bad and the entry is skipped.  The code words of a tile are stored transposed
+// (word k of chain slot j at (k * 128 + j) * 4) and every chain has `n_words` of them (<= 3, padded
+// with zero bytes = dummy points), so the loads are conflict free and the loop is warp-uniform.
+__device__ __forceinline__ void decode_chain(uint32_t stage, uint32_t wr, uint32_t hdr, uint32_t code_addr, uint32_t n_words, uint32_t* bad) {
   if (hdr == 0xFFFFFFFFu) return;                       // empty chain
   if (hdr & 0xE000E000u) { *bad = 1u; return; }
   uint32_t pos = hdr;
-  uint32_t word_addr = code_addr & ~3u;
-  const uint32_t shift = (code_addr & 3u) * 8u;
-  uint32_t w0 = 0, w1 = 0;
-  if (len != 0) { w0 = lds_u32(word_addr); w1 = lds_u32(word_addr + 4); }
+  uint32_t w[3] = {0u, 0u, 0u};
+#pragma unroll
+  for (int k = 0; k < 3; ++k)
+    if (static_cast<uint32_t>(k) < n_words) w[k] = lds_u32(code_addr + k * 512);
   {                                                     // first pair: absolute 16-bit positions
     const uint32_t off2 = swizzled_offset2(pos);
     const uint32_t at = stage + (off2 & 0xFFFFu);
@@ -313,41 +311,32 @@ __device__ __forceinline__ void decode_chain(uint32_t stage, uint32_t wr, uint32
     sts_u16(at, 0);                                     // W_t[offset_t] = 0
     sts_u16(wr + (off2 >> 16), v);                      // W_r[offset_r] = W_t[offset_t]
   }
-  for (uint32_t k0 = 0; k0 < len; k0 += 4) {            // four delta bytes = one (unaligned) code word
-    uint32_t bytes = __funnelshift_r(w0, w1, shift);
-    const uint32_t rem = len - k0;
-    if (rem > 4) {                                      // code word of the next round
-      word_addr += 4;
-      w0 = w1;
-      w1 = lds_u32(word_addr + 4);
-    } else if (rem < 4) {                               // bytes past the end behave like dummies
-      bytes &= (1u << (8 * rem)) - 1u;
+#pragma unroll
+  for (int k = 0; k < 3; ++k) {                         // one code word = four delta bytes
+    if (static_cast<uint32_t>(k) >= n_words) break;
+    const uint32_t bytes = w[k];
+    uint32_t off2[4], val[4];
+    bool real[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint32_t bt = __byte_perm(bytes, 0u, 0x4440u + q);    // delta byte q
+      const uint32_t delta = (bt * 0x1001u) & 0x000F000Fu;        // t delta | r delta << 16
+      pos += delta;
+      real[q] = ((delta - 0x00010001u) & 0x80008000u) == 0u;      // both nibbles non-zero (else a dummy point)
+      off2[q] = swizzled_offset2(pos);
+    }
+    // both cursors only grow, so the last position of the round bounds them all
+    if (pos & 0xE000E000u) {
+      *bad = 2u;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) real[q] = false;
     }
 #pragma unroll
-    for (int b0 = 0; b0 < 4; b0 += kBatch) {
-      uint32_t off2[kBatch], val[kBatch];
-      bool real[kBatch];
+    for (int q = 0; q < 4; ++q)
+      if (real[q]) val[q] = lds_u16(stage + (off2[q] & 0xFFFFu));
 #pragma unroll
-      for (int q = 0; q < kBatch; ++q) {
-        const uint32_t bt = __byte_perm(bytes, 0u, 0x4440u + b0 + q);   // delta byte b0 + q
-        const uint32_t delta = (bt * 0x1001u) & 0x000F000Fu;      // t delta | r delta << 16
-        pos += delta;
-        real[q] = ((delta - 0x00010001u) & 0x80008000u) == 0u;    // both nibbles non-zero (else a dummy point)
-        off2[q] = swizzled_offset2(pos);
-      }
-      // both cursors only grow, so the last position of the round bounds them all
-      if (pos & 0xE000E000u) {
-        *bad = 2u;
-#pragma unroll
-        for (int q = 0; q < kBatch; ++q) real[q] = false;
-      }
-#pragma unroll
-      for (int q = 0; q < kBatch; ++q)
-        if (real[q]) val[q] = lds_u16(stage + (off2[q] & 0xFFFFu));
-#pragma unroll
-      for (int q = 0; q < kBatch; ++q)
-        if (real[q]) { sts_u16(stage + (off2[q] & 0xFFFFu), 0); sts_u16(wr + (off2[q] >> 16), val[q]); }
-    }
+    for (int q = 0; q < 4; ++q)
+      if (real[q]) { sts_u16(stage + (off2[q] & 0xFFFFu), 0); sts_u16(wr + (off2[q] >> 16), val[q]); }
   }
 }
 
@@ -594,12 +583,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0, span = 0, hdr = 0xFFFFFFFFu, pdd_len = 0, res_cnt = 0;
       if (ok) {
         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(m0), "=r"(m1), "=r"(m2), "=r"(m3) : "r"(stage + kMetaOff + r * 16));
-        {
-          uint16_t o0, o1;
-          asm volatile("ld.shared.u16 %0, [%1];" : "=h"(o0) : "r"(stage + kLenOff + cr * 2));
-          asm volatile("ld.shared.u16 %0, [%1];" : "=h"(o1) : "r"(stage + kLenOff + cr * 2 + 2));
-          span = static_cast<uint32_t>(o0) | static_cast<uint32_t>(o1) << 16;
-        }
+        span = lds_u32(stage + kInfoOff + 8);                      // code words per chain
         hdr = lds_u32(stage + kHdrOff + cr * 4);
         pdd_len = lds_u32(stage + kInfoOff);
         res_cnt = lds_u32(stage + kInfoOff + 4);
@@ -611,14 +595,13 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
                      ::"r"(tmem_base + lane_base + kColMetaT + 4 * wb), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
       }
-      // byte offset and length of this thread's chain: the block lists where each chain's code starts
-      const uint32_t off = span & 0xFFFFu, len = (span >> 16) - off;
+      const uint32_t n_words = span;
       TL3_TACC(4)
       uint32_t bad = 0;
       const uint32_t room = a.x_offset - kPddOff;               // bytes a block may use after its fixed part
       const bool lens_ok = pdd_len <= room && res_cnt <= room / 4 && ((pdd_len + 3u) & ~3u) + 4u * res_cnt <= room &&
-                           (span >> 16) >= off && len <= 255u && off + len <= pdd_len;
-      if (lens_ok) decode_chain(stage, wr, hdr, stage + kPddOff + off, len, &bad);
+                           n_words <= 3u && pdd_len == n_words * 512u;
+      if (lens_ok) decode_chain(stage, wr, hdr, stage + kPddOff + cr * 4, n_words, &bad);
       else bad = 3u;
       __syncwarp();
       TL3_TACC(5)
@@ -975,8 +958,7 @@ static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, 
   const int n_pad = n_pad_of(N);
 
   // shared-memory plan
-  // + 48: the decoder fetches delta bytes in aligned words, one batch ahead, and may read that far past a block
-  const uint32_t block_area = (m->max_block_bytes + 48u + 1023u) / 1024u * 1024u;
+  const uint32_t block_area = (m->max_block_bytes + 1023u) / 1024u * 1024u;
   const uint32_t x_bytes = 128u * n_pad * 2u;
   const uint32_t stage_stride = block_area + x_bytes;
   // W_r ring of five buffers if that still leaves five stages, else four

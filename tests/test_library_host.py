@@ -161,7 +161,7 @@ def _decode_device_blob(blob, M_pad, K_pad):
         tm, tk = divmod(t, tiles_k)
         off16, nbytes, pdd_len, res_cnt = (int(x) for x in directory[t])
         assert (off16 * 16) % 128 == 0 and off16 * 16 >= seen_end             # aligned, no overlap
-        assert nbytes == (19224 + (pdd_len + 3) // 4 * 4 + 4 * res_cnt + 15) // 16 * 16
+        assert nbytes == (18960 + pdd_len + 4 * res_cnt + 15) // 16 * 16
         seen_end = off16 * 16 + nbytes
         blk = blob[off16 * 16: off16 * 16 + nbytes]
         img = blk[:16384].view(np.uint16).copy()                              # W_t image, halfword = byte offset / 2
@@ -169,20 +169,16 @@ def _decode_device_blob(blob, M_pad, K_pad):
         info = blk[18432:18448].view(np.uint32)
         assert (int(info[0]), int(info[1])) == (pdd_len, res_cnt)
         hdr = blk[18448:18960].view(np.uint32)
-        offs = blk[18960:18960 + 2 * 129].view(np.uint16).astype(np.int64)       # where each chain's code starts
-        assert offs[0] == 0 and offs[128] == pdd_len and (np.diff(offs) >= 0).all() and (np.diff(offs) <= 12).all()
-        lens = np.diff(offs)
-        codes = blk[19224:19224 + pdd_len]
-        res = blk[19224 + (pdd_len + 3) // 4 * 4:][:4 * res_cnt].view(np.uint32)
+        n_words = int(info[2])                                                 # code words per chain, transposed
+        assert n_words <= 3 and pdd_len == 512 * n_words
+        words = blk[18960:18960 + pdd_len].view(np.uint32).reshape(n_words, 128)
+        res = blk[18960 + pdd_len:][:4 * res_cnt].view(np.uint32)
         wr = np.zeros(8192, dtype=np.uint16)                                   # W_r image
-        at = 0
         for j in range(128):
-            n, h = int(lens[j]), int(hdr[j])
-            if j >= 32:
-                assert int(lens[j - 32]) >= n                                  # longest first within a bank
-            assert at == offs[j]
+            h = int(hdr[j])
+            code = np.ascontiguousarray(words[:, j]).view(np.uint8)            # 4 * n_words delta bytes, zero padded
             if h == 0xFFFFFFFF:
-                assert n == 0
+                assert not code.any()
                 continue
             pt, pr = h & 0xFFFF, h >> 16
             assert pt < 8192 and pr < 8192 and (pt >> 8) == (j & 31)           # slot j: a chain of bank j % 32
@@ -196,14 +192,12 @@ def _decode_device_blob(blob, M_pad, K_pad):
                 wr[_image_offset(pr) // 2] = v
 
             move(pt, pr)
-            for b in codes[at:at + n]:
+            for b in code:
                 dt, dr = int(b) & 15, int(b) >> 4
-                assert dt or dr
                 pt += dt
                 pr += dr
                 if dt and dr:
                     move(pt, pr)
-            at += n
         for e in res:
             u, v = int(e) & 0xFFFF, int(e) >> 16
             assert u < 8192 and wr[_image_offset(u) // 2] == 0
@@ -239,8 +233,7 @@ def _decode_device_blob(blob, M_pad, K_pad):
 def test_device_blob_decodes_to_the_matrix(tl3, shape, sparsity, mask):
     """The packed device image (bank-major re-pairing of the Slot-Filling layer) holds the same
     matrix: an independent numpy decoder of the blob reproduces W bit for bit, every chain lies in
-    the bank of its lane, chains are longest first, and the blob is hardly larger than the
-    canonical container."""
+    the bank of its lane, and the blob is hardly larger than the canonical container."""
     M, K = shape
     W = wl.Case(0, "pack", M, K, 8, 9, sparsity, mask).make_W()
     m = tl3.encode(W)
