@@ -141,6 +141,20 @@ int tl3_workspace_init(void* workspace, size_t bytes, void* stream);
 int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N,
              void* workspace, void* stream);
 
+/* (No counterpart in the paper: the usual fused epilogue of a linear layer.)  Y = act(W X + b):
+ * tl3_spmm with a per-row bias and an activation applied to the fp32 sums before they are rounded
+ * to fp16.
+ *   ep->bias: device, fp16[M], or NULL for none.  ep->activation: TL3_ACT_NONE, TL3_ACT_RELU,
+ *   TL3_ACT_SILU (x / (1 + exp(-x))), TL3_ACT_GELU_TANH (0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))).
+ *   ep == NULL is tl3_spmm.  Everything else as for tl3_spmm; INVALID_ARG for an unknown activation. */
+enum { TL3_ACT_NONE = 0, TL3_ACT_RELU = 1, TL3_ACT_SILU = 2, TL3_ACT_GELU_TANH = 3 };
+typedef struct {
+  const void* bias;
+  int activation;
+} tl3_epilogue;
+int tl3_spmm_ex(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N,
+                const tl3_epilogue* ep, void* workspace, void* stream);
+
 /* Same product with HOST buffers: copies X to dX, runs tl3_spmm, copies dY to Y and waits for the
  * stream.  X, Y: host (pinned memory makes the copies asynchronous), dense leading dimensions
  * ldx = ldy = N.  dX (>= K*N*2 bytes) and dY (>= M*N*2 bytes): device scratch owned by the caller. */

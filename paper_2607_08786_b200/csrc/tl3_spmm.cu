@@ -87,6 +87,8 @@ struct KernelArgs {
   int M, N;
   long long ldy;
   __half* Y;
+  const __half* bias;        // per output row, added before the activation (null: none)
+  int act;                   // TL3_ACT_*
   float* partials;           // [2 * gridDim.x][n_pad][128]
   unsigned int* counters;    // [tiles_m]
   unsigned int* status;      // status word
@@ -235,6 +237,17 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 // row * 128 + bank * 4 + slot-in-window * 2.  The packer orders both PDD streams by u and gives
 // lane l of a decode warp a chain whose empty slots all lie in bank l.
 __device__ __forceinline__ uint32_t swizzled_offset(uint32_t u) { return ((u & 0x7Fu) << 7) | ((u >> 6) & 0x7Eu); }
+
+// Epilogue of tl3_spmm_ex: y = act(sum + bias), in fp32, before the rounding to fp16.  A real
+// call, not inlined: it is used from many unrolled places, and a kernel image that grows by tens of
+// kilobytes costs every launch time at its start.
+__device__ __noinline__ float finish(float v, float bias, int act) {
+  v += bias;
+  if (act == TL3_ACT_RELU) return fmaxf(v, 0.f);
+  if (act == TL3_ACT_SILU) return v / (1.f + __expf(-v));
+  if (act == TL3_ACT_GELU_TANH) return 0.5f * v * (1.f + tanhf(0.7978845608f * (v + 0.044715f * v * v * v)));
+  return v;
+}
 
 template <int NPAD> struct TmemLd;
 template <> struct TmemLd<16> {
@@ -644,6 +657,9 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       const bool complete = (t == row_tile_begin) && (seg_end == row_tile_end);
       const int b = seg & 1;
       const int c_first = owner_of(row_tile_begin, T, G), c_last = owner_of(row_tile_end - 1, T, G);
+      const int row = mt * kTileM + et;
+      float bias_v = 0.f;                                         // fetched before the wait: off the tail of the segment
+      if (a.bias != nullptr && row < a.M) bias_v = __half2float(__ldg(a.bias + row));
       // A row-tile shared with other CTAs: look at its arrival counter before waiting for the
       // accumulator.  If every other contributor has arrived by then, this CTA is the last one: it
       // adds the others' partial sums to its own registers and writes Y directly, without the
@@ -659,19 +675,22 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       tc_fence_after();
       const bool all_others_in = !complete && *last_flag == 2u;
       constexpr int CH = NPAD < 32 ? NPAD : 32;                 // columns handled per round (register budget)
-      const int row = mt * kTileM + et;
       __half* y = a.Y + static_cast<long long>(row) * a.ldy;
-      const bool vec_ok = a.N == NPAD && (a.ldy & 7) == 0 && (reinterpret_cast<uintptr_t>(a.Y) & 15) == 0;
-      auto store_y = [&](const uint32_t* v, int c0) {           // fp32 -> fp16 (round to nearest even) -> Y
+      // 16-byte stores when the columns fill them (N = 8 runs in the 16-column kernel)
+      const bool vec_ok = (NPAD == 16 ? (a.N & 7) == 0 : a.N == NPAD) && (a.ldy & 7) == 0 && (reinterpret_cast<uintptr_t>(a.Y) & 15) == 0;
+      const bool plain = a.bias == nullptr && a.act == TL3_ACT_NONE;
+      auto fin = [&](uint32_t bits) { const float f = __uint_as_float(bits); return plain ? f : finish(f, bias_v, a.act); };
+      auto store_y = [&](const uint32_t* v, int c0) {           // (bias, activation,) fp32 -> fp16 (round to nearest even) -> Y
         if (row >= a.M) return;
         if (vec_ok) {
 #pragma unroll
           for (int c = 0; c < CH; c += 8) {
+            if (NPAD == 16 && c0 + c >= a.N) break;
             uint4 o;
-            __half2 h0 = __floats2half2_rn(__uint_as_float(v[c + 0]), __uint_as_float(v[c + 1]));
-            __half2 h1 = __floats2half2_rn(__uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
-            __half2 h2 = __floats2half2_rn(__uint_as_float(v[c + 4]), __uint_as_float(v[c + 5]));
-            __half2 h3 = __floats2half2_rn(__uint_as_float(v[c + 6]), __uint_as_float(v[c + 7]));
+            __half2 h0 = __floats2half2_rn(fin(v[c + 0]), fin(v[c + 1]));
+            __half2 h1 = __floats2half2_rn(fin(v[c + 2]), fin(v[c + 3]));
+            __half2 h2 = __floats2half2_rn(fin(v[c + 4]), fin(v[c + 5]));
+            __half2 h3 = __floats2half2_rn(fin(v[c + 6]), fin(v[c + 7]));
             o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
             o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
             *reinterpret_cast<uint4*>(y + c0 + c) = o;
@@ -679,7 +698,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         } else {
 #pragma unroll
           for (int c = 0; c < CH; ++c)
-            if (c0 + c < a.N) y[c0 + c] = __float2half_rn(__uint_as_float(v[c]));
+            if (c0 + c < a.N) y[c0 + c] = __float2half_rn(fin(v[c]));
         }
       };
       const uint32_t acc_tmem = tmem_base + lane_base + static_cast<uint32_t>(b * NPAD);
@@ -711,9 +730,12 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
             if (vec_ok) {
 #pragma unroll
               for (int c = 0; c < 16; c += 8) {
+                if (NPAD == 16 && c0 + c >= a.N) break;
                 uint4 o;
-                __half2 h0 = __floats2half2_rn(acc[c + 0], acc[c + 1]), h1 = __floats2half2_rn(acc[c + 2], acc[c + 3]);
-                __half2 h2 = __floats2half2_rn(acc[c + 4], acc[c + 5]), h3 = __floats2half2_rn(acc[c + 6], acc[c + 7]);
+                __half2 h0 = __floats2half2_rn(fin(__float_as_uint(acc[c + 0])), fin(__float_as_uint(acc[c + 1])));
+                __half2 h1 = __floats2half2_rn(fin(__float_as_uint(acc[c + 2])), fin(__float_as_uint(acc[c + 3])));
+                __half2 h2 = __floats2half2_rn(fin(__float_as_uint(acc[c + 4])), fin(__float_as_uint(acc[c + 5])));
+                __half2 h3 = __floats2half2_rn(fin(__float_as_uint(acc[c + 6])), fin(__float_as_uint(acc[c + 7])));
                 o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
                 o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
                 *reinterpret_cast<uint4*>(y + c0 + c) = o;
@@ -721,7 +743,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
             } else {
 #pragma unroll
               for (int c = 0; c < 16; ++c)
-                if (c0 + c < a.N) y[c0 + c] = __float2half_rn(acc[c]);
+                if (c0 + c < a.N) y[c0 + c] = __float2half_rn(fin(__float_as_uint(acc[c])));
             }
           }
         }
@@ -946,7 +968,7 @@ int tl3_workspace_init(void* workspace, size_t bytes, void* stream) {
 }
 
 // one launch: at most 64 columns
-static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N, void* workspace, void* stream) {
+static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N, const tl3_epilogue* ep, void* workspace, void* stream) {
   using namespace tl3;
   if (N < 1 || N > 64) return TL3_ERR_UNSUPPORTED;
   if (ldx < N || ldy < N || (ldx & 7) != 0 || (reinterpret_cast<uintptr_t>(X) & 15) != 0 ||
@@ -1001,6 +1023,8 @@ static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, 
   args.N = N;
   args.ldy = ldy;
   args.Y = static_cast<__half*>(Y);
+  args.bias = ep ? static_cast<const __half*>(ep->bias) : nullptr;
+  args.act = ep ? ep->activation : TL3_ACT_NONE;
   args.partials = reinterpret_cast<float*>(ws + wl.partials_off);
   args.counters = reinterpret_cast<unsigned int*>(ws + wl.counters_off);
   args.status = reinterpret_cast<unsigned int*>(ws + wl.status_off);
@@ -1023,7 +1047,15 @@ static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, 
 }
 
 int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N, void* workspace, void* stream) {
+  return tl3_spmm_ex(m, X, ldx, Y, ldy, N, nullptr, workspace, stream);
+}
+
+int tl3_spmm_ex(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N, const tl3_epilogue* ep,
+                void* workspace, void* stream) {
   if (!m || !X || !Y || !workspace) return TL3_ERR_INVALID_ARG;
+  if (ep && (ep->activation < TL3_ACT_NONE || ep->activation > TL3_ACT_GELU_TANH ||
+             (reinterpret_cast<uintptr_t>(ep->bias) & 1) != 0))
+    return TL3_ERR_INVALID_ARG;
   if (!m->dptr) return TL3_ERR_NOT_UPLOADED;
   if (N < 1 || N > TL3_MAX_N) return TL3_ERR_UNSUPPORTED;
   if (ldx < N || ldy < N) return TL3_ERR_INVALID_ARG;
@@ -1032,7 +1064,7 @@ int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t l
   // paper, too, loses to the dense GEMM at large N, Sec. 6).
   for (int n0 = 0; n0 < N; n0 += 64) {
     const int nb = N - n0 < 64 ? N - n0 : 64;
-    const int rc = spmm_block(m, static_cast<const uint16_t*>(X) + n0, ldx, static_cast<uint16_t*>(Y) + n0, ldy, nb, workspace, stream);
+    const int rc = spmm_block(m, static_cast<const uint16_t*>(X) + n0, ldx, static_cast<uint16_t*>(Y) + n0, ldy, nb, ep, workspace, stream);
     if (rc != TL3_OK) return rc;
   }
   return TL3_OK;

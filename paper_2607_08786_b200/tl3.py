@@ -27,7 +27,7 @@ _CANONICAL_DTYPES = (np.uint16, np.uint8, np.uint16, np.uint16, np.uint8, np.uin
 # every symbol include/tl3.h declares
 SYMBOLS = ("tl3_encode", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_deserialize",
            "tl3_free", "tl3_device_bytes", "tl3_pack", "tl3_upload", "tl3_workspace_bytes", "tl3_workspace_init",
-           "tl3_spmm", "tl3_spmm_host", "tl3_spmm_static_scratch", "tl3_static_scratch_status", "tl3_status", "tl3_status_word", "tl3_last_launch", "tl3_strerror",
+           "tl3_spmm", "tl3_spmm_ex", "tl3_spmm_host", "tl3_spmm_static_scratch", "tl3_static_scratch_status", "tl3_status", "tl3_status_word", "tl3_last_launch", "tl3_strerror",
            "tl3_last_cuda_error")
 
 
@@ -42,6 +42,13 @@ class Tl3Error(RuntimeError):
 
 class Params(ctypes.Structure):
     _fields_ = [("tile_m", ctypes.c_int32), ("tile_k", ctypes.c_int32), ("maxd", ctypes.c_int32)]
+
+
+class Epilogue(ctypes.Structure):
+    _fields_ = [("bias", ctypes.c_void_p), ("activation", ctypes.c_int32)]
+
+
+ACTIVATIONS = {None: 0, "none": 0, "relu": 1, "silu": 2, "gelu_tanh": 3}
 
 
 class Stats(ctypes.Structure):
@@ -81,6 +88,7 @@ def lib() -> ctypes.CDLL:
         L.tl3_workspace_bytes.restype = sz
         L.tl3_workspace_init.argtypes = [vp, sz, vp]
         L.tl3_spmm.argtypes = [vp, vp, i64, vp, i64, ci, vp, vp]
+        L.tl3_spmm_ex.argtypes = [vp, vp, i64, vp, i64, ci, ctypes.POINTER(Epilogue), vp, vp]
         L.tl3_spmm_host.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp]
         L.tl3_spmm_static_scratch.argtypes = [vp, vp, i64, vp, i64, ci, vp]
         L.tl3_static_scratch_status.argtypes = [vp]
@@ -222,8 +230,10 @@ class Matrix:
         _check(lib().tl3_workspace_init(ws.data_ptr(), n, _stream_ptr(stream)), "tl3_workspace_init")
         return ws
 
-    def spmm(self, X, Y=None, workspace=None, stream=None):
-        """``Y = W X`` on the GPU.  X: torch.float16 (K x N, last dim contiguous) on the device."""
+    def spmm(self, X, Y=None, workspace=None, stream=None, bias=None, activation=None):
+        """``Y = W X`` on the GPU, or ``Y = act(W X + bias)`` when a bias (torch.float16, M entries, on
+        the device) and / or an activation ("relu", "silu", "gelu_tanh") is given.
+        X: torch.float16 (K x N, last dim contiguous) on the device."""
         import torch
         if X.dtype != torch.float16 or X.dim() != 2 or X.stride(1) != 1:
             raise ValueError("X must be a 2-D float16 tensor with contiguous rows")
@@ -238,8 +248,15 @@ class Matrix:
             workspace = self._workspaces.get(key)
             if workspace is None:
                 workspace = self._workspaces[key] = self.new_workspace(N, stream)
-        _check(lib().tl3_spmm(self._h, X.data_ptr(), X.stride(0), Y.data_ptr(), Y.stride(0), N,
-                              workspace.data_ptr(), _stream_ptr(stream)), "tl3_spmm")
+        if bias is None and activation is None:
+            _check(lib().tl3_spmm(self._h, X.data_ptr(), X.stride(0), Y.data_ptr(), Y.stride(0), N,
+                                  workspace.data_ptr(), _stream_ptr(stream)), "tl3_spmm")
+            return Y
+        if bias is not None and (bias.dtype != torch.float16 or bias.numel() != M or not bias.is_contiguous()):
+            raise ValueError("bias must be a contiguous float16 tensor with one entry per row of W")
+        ep = Epilogue(bias.data_ptr() if bias is not None else None, ACTIVATIONS[activation])
+        _check(lib().tl3_spmm_ex(self._h, X.data_ptr(), X.stride(0), Y.data_ptr(), Y.stride(0), N, ctypes.byref(ep),
+                                 workspace.data_ptr(), _stream_ptr(stream)), "tl3_spmm_ex")
         return Y
 
     def spmm_static_scratch(self, X, Y=None, stream=None):

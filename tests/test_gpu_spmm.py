@@ -226,6 +226,40 @@ def test_wide_activation_blocks(tl3, oracle_mod, N):
     check(oracle_mod, W, X, Y)
 
 
+@pytest.mark.parametrize("activation", [None, "relu", "silu", "gelu_tanh"])
+@pytest.mark.parametrize("shape", [(384, 512, 16), (1000, 1096, 24), (5120, 640, 32)])
+def test_bias_and_activation_epilogue(tl3, oracle_mod, activation, shape):
+    """Y = act(W X + b) against the same expression in float64 (complete row-tiles, the direct
+    write of the last contributor and the reduction of partial sums all pass through it)."""
+    import torch
+    M, K, N = shape
+    case = wl.Case(0, "ep", M, K, N, 31, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    bias = (np.random.default_rng(7).standard_normal(M) * 0.5).astype(np.float16)
+    m = tl3.encode(W)
+    m.upload()
+    Y = m.spmm(device_X(X), bias=torch.from_numpy(bias).cuda(), activation=activation)
+    torch.cuda.synchronize()
+    Yref, bound = oracle_mod.dense_fp64(W, X)
+    z = Yref + bias.astype(np.float64)[:, None]
+    if activation == "relu":
+        ref = np.maximum(z, 0)
+    elif activation == "silu":
+        ref = z / (1 + np.exp(-z))
+    elif activation == "gelu_tanh":
+        ref = 0.5 * z * (1 + np.tanh(np.sqrt(2 / np.pi) * (z + 0.044715 * z ** 3)))
+    else:
+        ref = z
+    # the activations used here have slopes within [-0.13, 1.13]; the output rounding is within the 1e-3 + 2e-3 * bound
+    tol = 1.2 * oracle_mod.tolerance(bound + np.abs(bias.astype(np.float64))[:, None]) + 1e-3
+    assert (np.abs(Y.cpu().numpy().astype(np.float64) - ref) <= tol).all()
+    if activation is None:                          # without a bias and an activation: the plain product, bit for bit
+        Y0 = m.spmm(device_X(X))
+        Y1 = m.spmm(device_X(X), bias=torch.zeros(M, dtype=torch.float16, device="cuda"))
+        torch.cuda.synchronize()
+        assert torch.equal(Y0, Y1)
+
+
 def test_strided_operands(tl3, oracle_mod):
     case = wl.Case(0, "ld", 300, 700, 12, 5, 0.5, "magnitude")
     W, X = case.make_W(), case.make_X()
