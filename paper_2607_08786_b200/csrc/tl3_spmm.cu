@@ -60,7 +60,7 @@ constexpr int kEpilogueWarp0 = kDecodeWarp0 + 4 * kGroups;
 constexpr int kThreads = (kEpilogueWarp0 + 4) * 32;
 constexpr int kMaxStages = 8;
 constexpr uint32_t kWrBytes = 16384;
-constexpr int kMaxWrBuffers = 5;          // W_r ring: tile i uses buffer i % num_wr (4 or 5, as shared memory allows)
+constexpr int kMaxWrBuffers = 5;          // W_r ring: tile i uses buffer i % num_wr (4 or 5, see the launcher)
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColMetaT = 128;       // + 4 * (W_r buffer): metadata of W_t, four columns per tile in flight
 constexpr uint32_t kColMetaR = 152;       // two columns of 0xEEEEEEEE
@@ -987,17 +987,23 @@ static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, 
   const uint32_t block_area = (m->max_block_bytes + 1023u) / 1024u * 1024u;
   const uint32_t x_bytes = 128u * n_pad * 2u;
   const uint32_t stage_stride = block_area + x_bytes;
-  // W_r ring of five buffers if that still leaves five stages, else four
+  // W_r ring of five buffers, or four if that makes room for one more stage (measured on
+  // 20480 x 5120, N = 16: 5 buffers + 5 stages 28.7 us, 4 + 6 28.1 us, 3 + 7 slower); the rest of
+  // the shared memory is stages
   int num_wr = kMaxWrBuffers, stages = 0;
   uint32_t fixed = 0;
-  for (;; --num_wr) {
-    fixed = num_wr * kWrBytes + kBarrierBytes + 1024u;          // + alignment slack
-    stages = fixed + stage_stride <= kSmemLimit ? static_cast<int>((kSmemLimit - fixed) / stage_stride) : 0;
-    if (stages >= 5 || num_wr == 4) break;
+  {
+    auto plan = [&](int nw) {
+      const uint32_t f = nw * kWrBytes + kBarrierBytes + 1024u;              // + alignment slack
+      return f + stage_stride <= kSmemLimit ? static_cast<int>((kSmemLimit - f) / stage_stride) : 0;
+    };
+    const int s5 = plan(kMaxWrBuffers), s4 = plan(4);
+    if (s4 > s5 && s5 < kMaxStages) num_wr = 4;
+    stages = num_wr == 4 ? s4 : s5;
+    fixed = num_wr * kWrBytes + kBarrierBytes + 1024u;
   }
   if (stages < 2) return TL3_ERR_UNSUPPORTED;
   if (stages > kMaxStages) stages = kMaxStages;
-  if (num_wr == kMaxWrBuffers && stages > 5) stages = 5;        // a sixth stage measured no faster than five
   const uint32_t smem_bytes = fixed + static_cast<uint32_t>(stages) * stage_stride;
 
   // tensor map of X: dims {N, K}, box {n_pad, 128}; columns >= N and rows >= K read as zero
