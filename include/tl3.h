@@ -155,6 +155,14 @@ typedef struct {
 int tl3_spmm_ex(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N,
                 const tl3_epilogue* ep, void* workspace, void* stream);
 
+/* The same product with both activations transposed, the [batch, hidden] layout of an inference
+ * stack (Sec. 2.1): Yt = Xt W^T, i.e. Yt[n][m] = sum_k W[m][k] Xt[n][k] (+ bias[m], activation).
+ *   Xt: device, fp16, N x K row-major, leading dimension ldxt >= K, ldxt % 8 == 0, 16-byte aligned.
+ *   Yt: device, fp16, N x M row-major, leading dimension ldyt >= M; rows 0..N-1 fully overwritten.
+ *   ep: as for tl3_spmm_ex, or NULL.  Everything else as for tl3_spmm. */
+int tl3_spmm_nt(const tl3_matrix* m, const void* Xt, int64_t ldxt, void* Yt, int64_t ldyt, int N,
+                const tl3_epilogue* ep, void* workspace, void* stream);
+
 /* Same product with HOST buffers: copies X to dX, runs tl3_spmm, copies dY to Y and waits for the
  * stream.  X, Y: host (pinned memory makes the copies asynchronous), dense leading dimensions
  * ldx = ldy = N.  dX (>= K*N*2 bytes) and dY (>= M*N*2 bytes): device scratch owned by the caller. */

@@ -357,7 +357,10 @@ __device__ __forceinline__ void decode_chain(uint32_t stage, uint32_t wr, uint32
   }
 }
 
-template <int NPAD>
+// XT: the activations are given as X^T (N x K row-major, the [batch, hidden] layout of an inference
+// stack, Sec. 2.1) and the result is written as Y^T (N x M row-major).  The X tile then arrives as
+// two boxes of 64 k-values (128 bytes per row, 128-byte swizzle) and is a K-major B operand.
+template <int NPAD, bool XT>
 __global__ void __launch_bounds__(kThreads, 1)
 tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   extern __shared__ uint8_t smem_raw[];
@@ -466,7 +469,12 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
             mbar_arrive_expect_tx(full, bytes + 128u * NPAD * 2u);
             bulk_copy_g2s(stage, src, bytes, full);
           }
-          tma_load_2d(stage + a.x_offset, &x_map, 0, kt * kTileK, full);
+          if (XT) {
+            tma_load_2d(stage + a.x_offset, &x_map, kt * kTileK, 0, full);
+            tma_load_2d(stage + a.x_offset + NPAD * 128u, &x_map, kt * kTileK + 64, 0, full);
+          } else {
+            tma_load_2d(stage + a.x_offset, &x_map, 0, kt * kTileK, full);
+          }
           TL3_STAMP(i, 1)
         }
         __syncwarp();
@@ -512,7 +520,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     // ------------------------------------------------------------------ MMA issuer
     // Warp-uniform loop; one elected lane issues the eight MMAs of a tile and the commits.
     // instruction descriptor: sparse, D = f32, A = B = f16, A K-major, B MN-major, N = NPAD, M = 128
-    const uint32_t idesc = (1u << 2) | (1u << 4) | (1u << 16) | (static_cast<uint32_t>(NPAD >> 3) << 17) | (8u << 24);
+    const uint32_t idesc = (1u << 2) | (1u << 4) | (XT ? 0u : (1u << 16)) | (static_cast<uint32_t>(NPAD >> 3) << 17) | (8u << 24);
     // Shared-memory descriptors: low word = start address >> 4 (+ an unused leading-offset field),
     // high word = stride between 8-row groups, descriptor version, swizzle mode.
     // A: K-major, 128-byte swizzle, 8-row groups 1024 B apart; a 32-wide k-block is 32 bytes of a row.
@@ -520,9 +528,15 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     //    a k-block is 32 rows.
     constexpr uint32_t kAHi = (1024u >> 4) | (1u << 14) | (2u << 29);
     constexpr uint32_t kBLayout = NPAD == 16 ? 6u : NPAD == 32 ? 4u : 2u;
-    constexpr uint32_t kBHi = ((8u * NPAD * 2u) >> 4) | (1u << 14) | (kBLayout << 29);
+    //    With XT: two sub-tiles of NPAD rows x 128 bytes (64 k-values each), K-major, 128-byte swizzle,
+    //    8-row groups 1024 B apart; a k-block is 64 bytes of a row.
+    constexpr uint32_t kBHi = XT ? ((1024u >> 4) | (1u << 14) | (2u << 29)) : (((8u * NPAD * 2u) >> 4) | (1u << 14) | (kBLayout << 29));
     constexpr uint32_t kLboOne = 1u << 16;
-    constexpr uint32_t kAStep = 32u >> 4, kBStep = (32u * NPAD * 2u) >> 4;
+    constexpr uint32_t kAStep = 32u >> 4;
+    auto b_step = [](int kb) -> uint32_t {                       // descriptor offset of k-block kb inside the X tile
+      return XT ? ((static_cast<uint32_t>(kb >> 1) * (NPAD * 128u) + static_cast<uint32_t>(kb & 1) * 64u) >> 4)
+                : (static_cast<uint32_t>(kb) * ((32u * NPAD * 2u) >> 4));
+    };
     const uint32_t a_lo0 = (smem_base >> 4) | kLboOne, stride16 = a.stage_stride >> 4, x16 = a.x_offset >> 4;
     const uint32_t w_lo0 = (smem_u32(wr_base) >> 4) | kLboOne;
     int seg = 0, s = 0, kt = kt_begin, wb = 0;
@@ -548,9 +562,9 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb) {
           const uint32_t id = idesc | static_cast<uint32_t>(kb & 1);
-          umma_sp_f16(d_tmem, a_lo + kb * kAStep, kAHi, b_lo + kb * kBStep, kBHi, e_t + (kb & ~1), id,
+          umma_sp_f16(d_tmem, a_lo + kb * kAStep, kAHi, b_lo + b_step(kb), kBHi, e_t + (kb & ~1), id,
                       (first_of_seg && kb == 0) ? 0u : 1u);
-          umma_sp_f16(d_tmem, w_lo + kb * kAStep, kAHi, b_lo + kb * kBStep, kBHi, e_r, id, 1u);
+          umma_sp_f16(d_tmem, w_lo + kb * kAStep, kAHi, b_lo + b_step(kb), kBHi, e_r, id, 1u);
         }
         umma_commit(mma_bar);         // frees the stage
         umma_commit(wrfree_bar);      // frees this tile's W_r buffer and metadata columns
@@ -679,9 +693,9 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       tc_fence_after();
       const bool all_others_in = !complete && *last_flag == 2u;
       constexpr int CH = NPAD < 32 ? NPAD : 32;                 // columns handled per round (register budget)
-      __half* y = a.Y + static_cast<long long>(row) * a.ldy;
+      __half* y = XT ? a.Y + row : a.Y + static_cast<long long>(row) * a.ldy;   // XT: element (row, c) at y[c * ldy]
       // 16-byte stores when the columns fill them (N = 8 runs in the 16-column kernel)
-      const bool vec_ok = (NPAD == 16 ? (a.N & 7) == 0 : a.N == NPAD) && (a.ldy & 7) == 0 && (reinterpret_cast<uintptr_t>(a.Y) & 15) == 0;
+      const bool vec_ok = !XT && (NPAD == 16 ? (a.N & 7) == 0 : a.N == NPAD) && (a.ldy & 7) == 0 && (reinterpret_cast<uintptr_t>(a.Y) & 15) == 0;
       const bool plain = a.bias == nullptr && a.act == TL3_ACT_NONE;
       auto fin = [&](uint32_t bits) { const float f = __uint_as_float(bits); return plain ? f : finish(f, bias_v, a.act); };
       auto store_y = [&](const uint32_t* v, int c0) {           // (bias, activation,) fp32 -> fp16 (round to nearest even) -> Y
@@ -701,8 +715,16 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
           }
         } else {
 #pragma unroll
-          for (int c = 0; c < CH; ++c)
-            if (c0 + c < a.N) y[c0 + c] = __float2half_rn(fin(v[c]));
+          if (XT) {
+            __half* yc = y + static_cast<long long>(c0) * a.ldy;          // column c0 of this row: Yt[c0][row]
+#pragma unroll
+            for (int c = 0; c < CH; ++c, yc += a.ldy)
+              if (c0 + c < a.N) *yc = __float2half_rn(fin(v[c]));
+          } else {
+#pragma unroll
+            for (int c = 0; c < CH; ++c)
+              if (c0 + c < a.N) y[c0 + c] = __float2half_rn(fin(v[c]));
+          }
         }
       };
       const uint32_t acc_tmem = tmem_base + lane_base + static_cast<uint32_t>(b * NPAD);
@@ -746,8 +768,16 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
               }
             } else {
 #pragma unroll
-              for (int c = 0; c < 16; ++c)
-                if (c0 + c < a.N) y[c0 + c] = __float2half_rn(fin(__float_as_uint(acc[c])));
+              if (XT) {
+                __half* yc = y + static_cast<long long>(c0) * a.ldy;
+#pragma unroll
+                for (int c = 0; c < 16; ++c, yc += a.ldy)
+                  if (c0 + c < a.N) *yc = __float2half_rn(fin(__float_as_uint(acc[c])));
+              } else {
+#pragma unroll
+                for (int c = 0; c < 16; ++c)
+                  if (c0 + c < a.N) y[c0 + c] = __float2half_rn(fin(__float_as_uint(acc[c])));
+              }
             }
           }
         }
@@ -902,11 +932,11 @@ static WorkspaceLayout workspace_layout(const tl3_matrix* m, int n_pad, int sm_c
   return w;
 }
 
-template <int NPAD>
+template <int NPAD, bool XT>
 static int launch(const CUtensorMap& map, const KernelArgs& args, int grid, uint32_t smem_bytes, cudaStream_t stream) {
   static bool configured = false;   // per template instance; same value every time
   if (!configured) {
-    TL3_CUDA(cudaFuncSetAttribute(tl3_spmm_kernel<NPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemLimit)));
+    TL3_CUDA(cudaFuncSetAttribute(tl3_spmm_kernel<NPAD, XT>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemLimit)));
     configured = true;
   }
   cudaLaunchConfig_t cfg = {};
@@ -919,7 +949,7 @@ static int launch(const CUtensorMap& map, const KernelArgs& args, int grid, uint
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  TL3_CUDA(cudaLaunchKernelEx(&cfg, tl3_spmm_kernel<NPAD>, map, args));
+  TL3_CUDA(cudaLaunchKernelEx(&cfg, tl3_spmm_kernel<NPAD, XT>, map, args));
   TL3_CUDA(cudaGetLastError());
   return TL3_OK;
 }
@@ -972,10 +1002,12 @@ int tl3_workspace_init(void* workspace, size_t bytes, void* stream) {
 }
 
 // one launch: at most 64 columns
-static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N, const tl3_epilogue* ep, void* workspace, void* stream) {
+// (xt: X and Y are given transposed, N x K and N x M row-major)
+static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N, const tl3_epilogue* ep, bool xt,
+                      void* workspace, void* stream) {
   using namespace tl3;
   if (N < 1 || N > 64) return TL3_ERR_UNSUPPORTED;
-  if (ldx < N || ldy < N || (ldx & 7) != 0 || (reinterpret_cast<uintptr_t>(X) & 15) != 0 ||
+  if (ldx < (xt ? m->K : N) || ldy < (xt ? m->M : N) || (ldx & 7) != 0 || (reinterpret_cast<uintptr_t>(X) & 15) != 0 ||
       (reinterpret_cast<uintptr_t>(Y) & 1) != 0 || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0)
     return TL3_ERR_INVALID_ARG;
   DeviceInfo di;
@@ -1010,11 +1042,13 @@ static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, 
   EncodeTiledFn encode = encode_tiled_fn();
   if (!encode) return TL3_ERR_UNSUPPORTED;
   CUtensorMap map;
-  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(m->K)};
+  // (transposed: dims {K, N}, box {64, n_pad}, two boxes per tile)
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(xt ? m->K : N), static_cast<cuuint64_t>(xt ? N : m->K)};
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ldx) * 2};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(n_pad), 128};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(xt ? 64 : n_pad), static_cast<cuuint32_t>(xt ? n_pad : 128)};
   const cuuint32_t elem_strides[2] = {1, 1};
-  const CUtensorMapSwizzle swz = n_pad == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : n_pad == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
+  const CUtensorMapSwizzle swz = xt ? CU_TENSOR_MAP_SWIZZLE_128B
+                               : n_pad == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : n_pad == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
   const CUresult cr = encode(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(X), dims, strides, box, elem_strides,
                              CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (cr != CUDA_SUCCESS) { set_cuda_error(static_cast<int>(cr)); return TL3_ERR_CUDA; }
@@ -1049,10 +1083,17 @@ static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, 
 #endif
   m->last_ctas = grid; m->last_stages = stages; m->last_smem = static_cast<int>(smem_bytes);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (xt) {
+    switch (n_pad) {
+      case 16: return launch<16, true>(map, args, grid, smem_bytes, st);
+      case 32: return launch<32, true>(map, args, grid, smem_bytes, st);
+      default: return launch<64, true>(map, args, grid, smem_bytes, st);
+    }
+  }
   switch (n_pad) {
-    case 16: return launch<16>(map, args, grid, smem_bytes, st);
-    case 32: return launch<32>(map, args, grid, smem_bytes, st);
-    default: return launch<64>(map, args, grid, smem_bytes, st);
+    case 16: return launch<16, false>(map, args, grid, smem_bytes, st);
+    case 32: return launch<32, false>(map, args, grid, smem_bytes, st);
+    default: return launch<64, false>(map, args, grid, smem_bytes, st);
   }
 }
 
@@ -1074,7 +1115,25 @@ int tl3_spmm_ex(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_
   // paper, too, loses to the dense GEMM at large N, Sec. 6).
   for (int n0 = 0; n0 < N; n0 += 64) {
     const int nb = N - n0 < 64 ? N - n0 : 64;
-    const int rc = spmm_block(m, static_cast<const uint16_t*>(X) + n0, ldx, static_cast<uint16_t*>(Y) + n0, ldy, nb, ep, workspace, stream);
+    const int rc = spmm_block(m, static_cast<const uint16_t*>(X) + n0, ldx, static_cast<uint16_t*>(Y) + n0, ldy, nb, ep, false, workspace, stream);
+    if (rc != TL3_OK) return rc;
+  }
+  return TL3_OK;
+}
+
+int tl3_spmm_nt(const tl3_matrix* m, const void* Xt, int64_t ldxt, void* Yt, int64_t ldyt, int N, const tl3_epilogue* ep,
+                void* workspace, void* stream) {
+  if (!m || !Xt || !Yt || !workspace) return TL3_ERR_INVALID_ARG;
+  if (ep && (ep->activation < TL3_ACT_NONE || ep->activation > TL3_ACT_GELU_TANH ||
+             (reinterpret_cast<uintptr_t>(ep->bias) & 1) != 0))
+    return TL3_ERR_INVALID_ARG;
+  if (!m->dptr) return TL3_ERR_NOT_UPLOADED;
+  if (N < 1 || N > TL3_MAX_N) return TL3_ERR_UNSUPPORTED;
+  if (ldxt < m->K || ldyt < m->M) return TL3_ERR_INVALID_ARG;
+  for (int n0 = 0; n0 < N; n0 += 64) {                           // 64 rows of X^T (= columns of X) per launch
+    const int nb = N - n0 < 64 ? N - n0 : 64;
+    const int rc = spmm_block(m, static_cast<const uint16_t*>(Xt) + static_cast<int64_t>(n0) * ldxt, ldxt,
+                              static_cast<uint16_t*>(Yt) + static_cast<int64_t>(n0) * ldyt, ldyt, nb, ep, true, workspace, stream);
     if (rc != TL3_OK) return rc;
   }
   return TL3_OK;

@@ -27,7 +27,7 @@ _CANONICAL_DTYPES = (np.uint16, np.uint8, np.uint16, np.uint16, np.uint8, np.uin
 # every symbol include/tl3.h declares
 SYMBOLS = ("tl3_encode", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_deserialize",
            "tl3_free", "tl3_device_bytes", "tl3_pack", "tl3_upload", "tl3_workspace_bytes", "tl3_workspace_init",
-           "tl3_spmm", "tl3_spmm_ex", "tl3_spmm_host", "tl3_spmm_static_scratch", "tl3_static_scratch_status", "tl3_status", "tl3_status_word", "tl3_last_launch", "tl3_strerror",
+           "tl3_spmm", "tl3_spmm_ex", "tl3_spmm_nt", "tl3_spmm_host", "tl3_spmm_static_scratch", "tl3_static_scratch_status", "tl3_status", "tl3_status_word", "tl3_last_launch", "tl3_strerror",
            "tl3_last_cuda_error")
 
 
@@ -89,6 +89,7 @@ def lib() -> ctypes.CDLL:
         L.tl3_workspace_init.argtypes = [vp, sz, vp]
         L.tl3_spmm.argtypes = [vp, vp, i64, vp, i64, ci, vp, vp]
         L.tl3_spmm_ex.argtypes = [vp, vp, i64, vp, i64, ci, ctypes.POINTER(Epilogue), vp, vp]
+        L.tl3_spmm_nt.argtypes = [vp, vp, i64, vp, i64, ci, ctypes.POINTER(Epilogue), vp, vp]
         L.tl3_spmm_host.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp]
         L.tl3_spmm_static_scratch.argtypes = [vp, vp, i64, vp, i64, ci, vp]
         L.tl3_static_scratch_status.argtypes = [vp]
@@ -258,6 +259,30 @@ class Matrix:
         _check(lib().tl3_spmm_ex(self._h, X.data_ptr(), X.stride(0), Y.data_ptr(), Y.stride(0), N, ctypes.byref(ep),
                                  workspace.data_ptr(), _stream_ptr(stream)), "tl3_spmm_ex")
         return Y
+
+    def spmm_nt(self, Xt, Yt=None, workspace=None, stream=None, bias=None, activation=None):
+        """``Yt = Xt W^T`` (+ bias, activation): activations in the [batch, hidden] layout.
+        Xt: torch.float16 (N x K, last dim contiguous) on the device; Yt: N x M."""
+        import torch
+        if Xt.dtype != torch.float16 or Xt.dim() != 2 or Xt.stride(1) != 1:
+            raise ValueError("Xt must be a 2-D float16 tensor with contiguous rows")
+        M, K = self.shape
+        N = Xt.shape[0]
+        if Xt.shape[1] != K:
+            raise ValueError("Xt has the wrong number of columns")
+        if Yt is None:
+            Yt = torch.empty((N, M), dtype=torch.float16, device=Xt.device)
+        if workspace is None:
+            key = 16 if N <= 16 else 32 if N <= 32 else 64
+            workspace = self._workspaces.get(key)
+            if workspace is None:
+                workspace = self._workspaces[key] = self.new_workspace(N, stream)
+        if bias is not None and (bias.dtype != torch.float16 or bias.numel() != M or not bias.is_contiguous()):
+            raise ValueError("bias must be a contiguous float16 tensor with one entry per row of W")
+        ep = Epilogue(bias.data_ptr() if bias is not None else None, ACTIVATIONS[activation])
+        _check(lib().tl3_spmm_nt(self._h, Xt.data_ptr(), Xt.stride(0), Yt.data_ptr(), Yt.stride(0), N, ctypes.byref(ep),
+                                 workspace.data_ptr(), _stream_ptr(stream)), "tl3_spmm_nt")
+        return Yt
 
     def spmm_static_scratch(self, X, Y=None, stream=None):
         """``Y = W X`` without a caller-supplied workspace and without any allocation inside the

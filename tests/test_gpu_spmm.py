@@ -260,6 +260,36 @@ def test_bias_and_activation_epilogue(tl3, oracle_mod, activation, shape):
         assert torch.equal(Y0, Y1)
 
 
+@pytest.mark.parametrize("shape", [(384, 512, 16), (1000, 1096, 5), (130, 260, 24), (5120, 640, 32), (256, 4096, 64), (640, 896, 100)])
+def test_transposed_activations(tl3, oracle_mod, shape):
+    """Yt = Xt W^T with X and Y in the [batch, hidden] layout: the same numbers as Y = W X, and bit
+    for bit the same as the untransposed entry point (same products, same order)."""
+    import torch
+    M, K, N = shape
+    case = wl.Case(0, "nt", M, K, N, 41, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    m = tl3.encode(W)
+    m.upload()
+    ldk = (K + 7) // 8 * 8
+    Xt = torch.zeros((N, ldk), dtype=torch.float16, device="cuda")[:, :K]
+    Xt.copy_(torch.from_numpy(np.ascontiguousarray(X.T)))
+    Ytbuf = torch.full((N, M + 3), float("nan"), dtype=torch.float16, device="cuda")
+    Yt = m.spmm_nt(Xt, Ytbuf[:, :M])
+    torch.cuda.synchronize()
+    assert torch.isnan(Ytbuf[:, M:]).all()
+    Y = Yt.cpu().numpy().T
+    check(oracle_mod, W, X, np.ascontiguousarray(Y))
+    Y0 = m.spmm(device_X(X))
+    torch.cuda.synchronize()
+    assert np.array_equal(Y0.cpu().numpy().view(np.uint16), np.ascontiguousarray(Y).view(np.uint16))
+    bias = (np.random.default_rng(9).standard_normal(M) * 0.5).astype(np.float16)
+    b = torch.from_numpy(bias).cuda()
+    Y1 = m.spmm_nt(Xt, bias=b, activation="silu")
+    Y2 = m.spmm(device_X(X), bias=b, activation="silu")
+    torch.cuda.synchronize()
+    assert torch.equal(Y1.T.contiguous(), Y2)
+
+
 def test_strided_operands(tl3, oracle_mod):
     case = wl.Case(0, "ld", 300, 700, 12, 5, 0.5, "magnitude")
     W, X = case.make_W(), case.make_X()
