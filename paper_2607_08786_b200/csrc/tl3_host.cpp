@@ -209,6 +209,26 @@ bool consistent(const tl3_matrix& m) {
     uint64_t len_sum = 0;
     for (int r = 0; r < m.p.tile_m; ++r) len_sum += m.chain_len[t * m.p.tile_m + r];
     if (len_sum != d[1]) return false;
+    // every position a chain reaches lies inside the tile (the device packer and the decoders
+    // index with them)
+    uint64_t at = d[0];
+    for (int r = 0; r < m.p.tile_m; ++r) {
+      const size_t c = static_cast<size_t>(t) * m.p.tile_m + r;
+      uint32_t tau = m.chain_tau0[c], rho = m.chain_rho0[c];
+      const uint32_t len = m.chain_len[c];
+      if (tau == 0xFFFFu || rho == 0xFFFFu) {
+        if (tau != rho || len != 0) return false;
+        continue;
+      }
+      if (tau >= tile_slots || rho >= tile_slots) return false;
+      for (uint32_t k = 0; k < len; ++k) {
+        const uint32_t b = m.pdd_bytes[at + k];
+        tau += b & 15u;
+        rho += b >> 4;
+        if (tau >= tile_slots || rho >= tile_slots) return false;
+      }
+      at += len;
+    }
     for (uint32_t j = d[2]; j < d[2] + d[3]; ++j)
       if (m.res_rho[j] >= tile_slots) return false;
   }

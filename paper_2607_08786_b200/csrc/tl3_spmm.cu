@@ -714,7 +714,6 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
             *reinterpret_cast<uint4*>(y + c0 + c) = o;
           }
         } else {
-#pragma unroll
           if (XT) {
             __half* yc = y + static_cast<long long>(c0) * a.ldy;          // column c0 of this row: Yt[c0][row]
 #pragma unroll
@@ -767,7 +766,6 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
                 *reinterpret_cast<uint4*>(y + c0 + c) = o;
               }
             } else {
-#pragma unroll
               if (XT) {
                 __half* yc = y + static_cast<long long>(c0) * a.ldy;
 #pragma unroll

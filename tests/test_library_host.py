@@ -119,6 +119,26 @@ def test_corrupted_containers_are_rejected(tl3):
     blob[at:at + 2] = (0xFFFF).to_bytes(2, "little")
     with pytest.raises(tl3.Tl3Error):
         tl3.Matrix.deserialize(bytes(blob))
+    # a chain that runs out of its tile: a start beyond the last slot, and a delta byte that pushes it over
+    m = tl3.encode(CASES[0].make_W())
+    good = bytes(m.serialize())
+    tau0 = m.canonical("chain_tau0")
+    at = good.find(tau0.tobytes())
+    assert at > 0 and tau0[0] != 0xFFFF
+    bad = bytearray(good)
+    bad[at:at + 2] = (8192).to_bytes(2, "little")
+    with pytest.raises(tl3.Tl3Error) as e:
+        tl3.Matrix.deserialize(bytes(bad))
+    assert e.value.code == tl3.ERR_BAD_CONTAINER
+    pdd = m.canonical("pdd_bytes")
+    at = good.find(pdd.tobytes())
+    assert at > 0
+    bad = bytearray(good)
+    last_chain = int(np.flatnonzero(m.canonical("chain_len"))[-1])          # a chain near the end of a tile
+    bad[at:at + pdd.size] = b"\xFF" * pdd.size                              # every delta 15 + 15
+    with pytest.raises(tl3.Tl3Error):
+        tl3.Matrix.deserialize(bytes(bad))
+    assert last_chain >= 0
 
 
 def test_error_codes(tl3):
