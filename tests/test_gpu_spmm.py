@@ -136,6 +136,22 @@ def test_degenerate_matrices(tl3, oracle_mod):
     check(oracle_mod, T, X, Y)
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_adversarial_density_patterns(tl3, oracle_mod, seed):
+    """Density that changes abruptly by row band and column band: tiles with no parked elements,
+    tiles that are all Residual, tiles with one, two or three code words per chain, side by side."""
+    rng = np.random.default_rng([78, seed])
+    M, K, N = 640, 1152, (8, 16, 24, 32, 48, 64)[seed]
+    dens_r = rng.choice([0.0, 0.1, 0.5, 0.9, 1.0], size=M // 32).repeat(32)
+    dens_c = rng.choice([0.0, 0.25, 0.5, 0.75, 1.0], size=K // 64).repeat(64)
+    p = np.clip(0.5 * (dens_r[:, None] + dens_c[None, :]) + rng.choice([-0.3, 0.0, 0.3]), 0, 1)
+    W = np.where(rng.random((M, K)) < p, (rng.standard_normal((M, K)) * 0.05).astype(np.float16), np.float16(0))
+    W[(W.view(np.uint16) & 0x7FFF) == 0] = 0
+    X = rng.standard_normal((K, N)).astype(np.float16)
+    Y, _ = run_gpu(tl3, W, X, repeats=2)
+    check(oracle_mod, W, X, Y)
+
+
 def test_device_chain_overflow(tl3, oracle_mod):
     """A tile whose device-image chains overflow into the Residual list (see special_cases)."""
     from special_cases import clustered_surplus_tile

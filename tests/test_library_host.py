@@ -266,6 +266,26 @@ def test_device_blob_decodes_to_the_matrix(tl3, shape, sparsity, mask):
     assert np.array_equal(_decode_device_blob(blob, st["M_pad"], st["K_pad"]), ref)
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_device_blob_on_adversarial_patterns(tl3, seed):
+    """Tiles whose density changes abruptly by row band and by column band (empty bands, dense
+    bands, bands with only surplus or only empty slots): the packer's proportional selection of
+    empty slots, its equal-count chains and its cut after three code words must still give a blob
+    that decodes to the matrix."""
+    rng = np.random.default_rng([77, seed])
+    M, K = 256, 384
+    dens_r = rng.choice([0.0, 0.1, 0.5, 0.9, 1.0], size=M // 32).repeat(32)
+    dens_c = rng.choice([0.0, 0.25, 0.5, 0.75, 1.0], size=K // 64).repeat(64)
+    p = np.clip(0.5 * (dens_r[:, None] + dens_c[None, :]) + rng.choice([-0.3, 0.0, 0.3]), 0, 1)
+    W = np.where(rng.random((M, K)) < p, (rng.standard_normal((M, K)) * 0.05).astype(np.float16), np.float16(0))
+    W[(W.view(np.uint16) & 0x7FFF) == 0] = 0
+    m = tl3.encode(W)
+    st = m.stats()
+    blob = m.pack()
+    assert np.array_equal(_decode_device_blob(blob, st["M_pad"], st["K_pad"]), W.view(np.uint16))
+    assert np.array_equal(m.decode(), W.view(np.uint16))
+
+
 def test_device_chain_overflow_goes_to_the_residual_list(tl3):
     """A chain of the device image is cut when it is full (here: because two consecutive pairs lie
     thousands of positions apart); what is cut off travels in the Residual list, and the blob
