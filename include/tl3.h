@@ -118,10 +118,11 @@ int tl3_pack(const tl3_matrix* m, void* host_buf, size_t bytes);
  * Errors: UNSUPPORTED (tile shape other than 128 x 128), INVALID_ARG, CUDA. */
 int tl3_upload(tl3_matrix* m, void* dptr, void* stream);
 
-/* Scratch the kernel needs for N columns: split-K partial sums, arrival counters, a status word.
- * Depends on the current device's SM count.  The caller allocates it (device, 256-byte aligned),
- * clears it once with tl3_workspace_init(), and may then reuse it for any number of calls that
- * do not overlap on the GPU (the kernel leaves it cleared). */
+/* Scratch the kernel needs for N columns: split-K partial sums, one arrival flag per partial-sum
+ * slot, a status word.  Depends on the current device's SM count.  The caller allocates it (device,
+ * 256-byte aligned), clears it once with tl3_workspace_init(), and may then reuse it for any number
+ * of calls that do not overlap on the GPU (the kernel leaves it cleared; after a call that ended
+ * with a non-zero status, clear it again). */
 size_t tl3_workspace_bytes(const tl3_matrix* m, int N);
 int tl3_workspace_init(void* workspace, size_t bytes, void* stream);
 
@@ -173,7 +174,7 @@ int tl3_spmm_host(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int N, vo
  * not allowed to obtain device memory themselves and so cannot provide a workspace: a driver-level
  * plug-in whose host application hands it only the input and output buffers and forbids allocation
  * calls inside its execute hook, or a process running under a fixed device-memory budget that was
- * spent before this library was loaded.  The split-K partial sums, the arrival counters and the
+ * spent before this library was loaded.  The split-K partial sums, the arrival flags and the
  * status word live in a fixed array that is part of the library image: TL3_STATIC_SCRATCH_BYTES
  * (3 MiB) of device memory on every GPU that loads the library, held until the process exits.
  *   - Problems whose scratch need (what tl3_workspace_bytes() reports) exceeds that size are refused
@@ -183,7 +184,7 @@ int tl3_spmm_host(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int N, vo
  *   - The first call on each device looks up the array's device address (that device must be
  *     current); make that first call outside any stream capture.  Later calls only enqueue work.
  *   - The function calls no cudaMalloc / cudaFree nor any allocating routine, on any call.
- *   - All calls on a device share the one array.  Each call clears the counters and the status word
+ *   - All calls on a device share the one array.  Each call clears the flags and the status word
  *     on `stream` before the kernel, so a call that was cut short does not poison the next one, but
  *     two calls that overlap on the GPU (different streams, no dependency) race on it: serialise
  *     them.  tl3_static_scratch_status() reads the status word of the current device. */
@@ -196,7 +197,7 @@ int tl3_static_scratch_status(void* stream);
  * wait inside a kernel expired since the last tl3_workspace_init(); BAD_CONTAINER if the decoder
  * met a block whose lengths or decoded positions were out of range (it skips such entries rather
  * than touching memory outside the tile).  tl3_status_word() also hands back the raw word:
- * bits 0-7 = code (1-9: which wait gave up, 16: bad block), higher bits = detail. */
+ * bits 0-7 = code (1-11: which wait gave up, 16: bad block), higher bits = detail. */
 int tl3_status(const tl3_matrix* m, void* workspace, void* stream);
 int tl3_status_word(void* workspace, void* stream, uint32_t* word);
 

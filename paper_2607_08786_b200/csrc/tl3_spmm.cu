@@ -16,8 +16,9 @@
 //   * one thread issues tcgen05.mma.sp (kind::f16, M = 128, K = 32) on W_t and on W_r into the
 //     same fp32 accumulator in tensor memory (Sec. 4.3 "Sparse TC Computation");
 //   * four epilogue warps read the accumulator; a row-tile owned by one CTA is written to Y
-//     directly, otherwise partial sums go to the workspace and the last CTA to arrive adds them in
-//     a fixed order (Sec. 4.4: a single reduction at the end of the pipeline).
+//     directly, otherwise the CTAs that share it store partial sums in the workspace and raise a
+//     flag each, and the CTA that owns the row-tile's first tile collects them as the flags come
+//     up and adds them in a fixed order (Sec. 4.4: a single reduction at the end of the pipeline).
 // Every wait is bounded: on expiry the CTA records a code in the workspace status word, stops
 // issuing work, waits for its copies in flight, frees its tensor memory and returns.
 #include <cuda.h>
@@ -75,7 +76,7 @@ constexpr uint32_t kTryWaitHintNs = TL3_TRYWAIT_HINT_NS;     // how long one bar
 // status codes written to the workspace status word (0 = ok)
 enum : uint32_t {
   kStProducer = 1, kStDecodeFull = 2, kStDecodeWrFree = 3, kStMmaDecoded = 4, kStMmaAccEmpty = 5,
-  kStEpilogueAccFull = 6, kStDrain = 7, kStClearWrFree = 8, kStDecodeWrReady = 9, kStEpilogueTail = 10,
+  kStEpilogueAccFull = 6, kStDrain = 7, kStClearWrFree = 8, kStDecodeWrReady = 9, kStEpilogueTail = 10, kStEpilogueFlags = 11,
   kStBadBlock = 16           // a block's lengths or a decoded position were out of range (+ detail in bits 8..)
 };
 
@@ -90,7 +91,7 @@ struct KernelArgs {
   const __half* bias;        // per output row, added before the activation (null: none)
   int act;                   // TL3_ACT_*
   float* partials;           // [2 * gridDim.x][n_pad][128]
-  unsigned int* counters;    // [tiles_m]
+  unsigned int* flags;       // [2 * gridDim.x] one per partial-sum slot: 1 = written and not yet collected
   unsigned int* status;      // status word
   uint32_t stage_stride;     // bytes per stage (block area + X tile), multiple of 1024
   uint32_t x_offset;         // offset of the X tile inside a stage, multiple of 1024
@@ -130,6 +131,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {   // more bytes to come, no arrival
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -375,7 +379,6 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26), bar_wrready = smem_u32(bars + 44), bar_wrfree = smem_u32(bars + 49);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 32);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 33);
-  volatile unsigned int* last_flag = reinterpret_cast<volatile unsigned int*>(bars + 34);
   const uint32_t bar_tail = smem_u32(bars + 36);               // partial sums fetched into the idle stages at the very end
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -665,7 +668,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     int seg = 0;
     long long t = t_begin;
-    pdl_wait();   // Y, the partial sums and the counters may still be in use by the previous kernel
+    pdl_wait();   // Y, the partial sums and their flags may still be in use by the previous kernel
     TL3_T0()
     while (t < t_end) {
       TL3_TACC(0)
@@ -678,20 +681,14 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       const int row = mt * kTileM + et;
       float bias_v = 0.f;                                         // fetched before the wait: off the tail of the segment
       if (a.bias != nullptr && row < a.M) bias_v = __half2float(__ldg(a.bias + row));
-      // A row-tile shared with other CTAs: look at its arrival counter before waiting for the
-      // accumulator.  If every other contributor has arrived by then, this CTA is the last one: it
-      // adds the others' partial sums to its own registers and writes Y directly, without the
-      // partial-sum store, fence and atomic on its way out (the usual case for the segment a CTA
-      // ends with, since the CTAs it shares that row-tile with finished their part earlier).
-      if (!complete && et == 0) {
-        unsigned int seen;
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.counters + mt) : "memory");
-        *last_flag = seen == static_cast<unsigned int>(c_last - c_first) ? 2u : 0u;
-      }
+      // A row-tile shared with other CTAs is finished by the CTA that owns its first tile.  That
+      // CTA's range ends inside the row-tile (else the row-tile would not be shared), so this is
+      // always the last segment it works on: nothing of its own is held up while it collects.
+      const bool reducer = !complete && static_cast<int>(blockIdx.x) == c_first;
+      const int n_others = c_last - c_first;
       if (!named_bar_all(1 + kGroups, 128, mbar_wait(bar_accfull + 8 * b, (seg >> 1) & 1, wctx, kStEpilogueAccFull))) break;
       TL3_TACC(1)
       tc_fence_after();
-      const bool all_others_in = !complete && *last_flag == 2u;
       constexpr int CH = NPAD < 32 ? NPAD : 32;                 // columns handled per round (register budget)
       __half* y = XT ? a.Y + row : a.Y + static_cast<long long>(row) * a.ldy;   // XT: element (row, c) at y[c * ldy]
       // 16-byte stores when the columns fill them (N = 8 runs in the 16-column kernel)
@@ -730,59 +727,85 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       // partial sums of a shared row-tile: slot 2*cta + (this row-tile is not the first one of my range)
       const int slot = 2 * blockIdx.x + (t_begin < row_tile_begin ? 1 : 0);
       float* mine = a.partials + static_cast<size_t>(slot) * NPAD * 128 + et;
-      if (all_others_in) {
-        __threadfence();                                          // the others' partial sums, after the counter
-#pragma unroll 1
-        for (int c0 = 0; c0 < NPAD; c0 += 16) {                   // 16 columns at a time (register budget)
-          uint32_t v[CH];                                         // (only the first 16 are used)
-          TmemLd<16>::ld(acc_tmem + c0, v);
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-          float acc[16];
-#pragma unroll
-          for (int c = 0; c < 16; ++c) acc[c] = 0.f;
-          for (int c_id = c_first; c_id <= c_last; ++c_id) {      // same fixed order as the reduction below
-            if (c_id == static_cast<int>(blockIdx.x)) {
-#pragma unroll
-              for (int c = 0; c < 16; ++c) acc[c] += __uint_as_float(v[c]);
-            } else {
-              const int sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
-              const float* p = a.partials + static_cast<size_t>(sl) * NPAD * 128 + et;
-#pragma unroll
-              for (int c = 0; c < 16; ++c) acc[c] += __ldcg(p + (c0 + c) * 128);
+      if (reducer) {
+        // The other contributors store their partial sums and then raise the flag of their slot.
+        // One warp watches the flags and requests a slot the moment its flag is up (bulk copy into
+        // the stages, idle by now), so that when the last contributor arrives only its slot is
+        // still to come.  The sum runs in ascending CTA order whatever the order of arrival: the
+        // result does not depend on timing.
+        constexpr uint32_t kSlotBytes = NPAD * 128u * 4u;
+        const bool staged = seg_end == t_end && static_cast<uint32_t>(n_others) * kSlotBytes <= static_cast<uint32_t>(S) * a.stage_stride;
+        bool ok = true;
+        if (et < 32) {
+          for (int base = 0; base < n_others && ok; base += 32) {
+            const int k = base + et;                              // this lane watches contributor c_first + 1 + k
+            bool pending = k < n_others;
+            int sl = 0;
+            if (pending) {
+              const int c_id = c_first + 1 + k;
+              sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
+            }
+            for (uint32_t it = 0; __any_sync(0xFFFFFFFFu, pending); ++it) {
+              if (pending) {
+                unsigned int up;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(up) : "l"(a.flags + sl) : "memory");
+                if (up != 0u) {
+                  pending = false;
+                  a.flags[sl] = 0u;                               // leave the workspace cleared
+                  if (staged) {
+                    fence_proxy_async_all();
+                    mbar_expect_tx(bar_tail, kSlotBytes);
+                    bulk_copy_g2s(smem_base + static_cast<uint32_t>(k) * kSlotBytes, a.partials + static_cast<size_t>(sl) * NPAD * 128, kSlotBytes, bar_tail);
+                  }
+                }
+              }
+              if ((it & 15u) == 15u) {
+                const bool out = *abort_flag != 0 || global_timer() - wctx.t0 > kWaitLimitNs;
+                if (__any_sync(0xFFFFFFFFu, out)) {
+                  if (et == 0) { atomicCAS(a.status, 0u, static_cast<uint32_t>(kStEpilogueFlags)); *abort_flag = 1; }
+                  ok = false;
+                  break;
+                }
+              }
             }
           }
-          if (row < a.M) {
-            if (vec_ok) {
+          __syncwarp();
+          if (staged && et == 0) mbar_arrive(bar_tail);           // the phase ends when every requested slot has landed
+        }
+        bool fetched = named_bar_all(1 + kGroups, 128, ok);
+        if (staged) {
+          if (fetched) {
+            fetched = mbar_wait(bar_tail, 0, wctx, kStEpilogueTail);
+          } else if (et == 0) {                                   // giving up: still no exit with copies in flight
+            for (uint32_t it = 0; it < (1u << 16) && !mbar_try_wait(bar_tail, 0); ++it) {}
+          }
+        }
+        if (fetched) {
+          if (!staged) __threadfence();                           // the others' partial sums, after their flags
+#pragma unroll 1
+          for (int c0 = 0; c0 < NPAD; c0 += CH) {
+            uint32_t v[CH];
+            TmemLd<CH>::ld(acc_tmem + c0, v);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            for (int k = 0; k < n_others; ++k) {                  // own part first (lowest CTA), then ascending
+              if (staged) {
+                const uint32_t p = smem_base + (static_cast<uint32_t>(k) * NPAD * 128u + static_cast<uint32_t>(et)) * 4u;
 #pragma unroll
-              for (int c = 0; c < 16; c += 8) {
-                if (NPAD == 16 && c0 + c >= a.N) break;
-                uint4 o;
-                __half2 h0 = __floats2half2_rn(fin(__float_as_uint(acc[c + 0])), fin(__float_as_uint(acc[c + 1])));
-                __half2 h1 = __floats2half2_rn(fin(__float_as_uint(acc[c + 2])), fin(__float_as_uint(acc[c + 3])));
-                __half2 h2 = __floats2half2_rn(fin(__float_as_uint(acc[c + 4])), fin(__float_as_uint(acc[c + 5])));
-                __half2 h3 = __floats2half2_rn(fin(__float_as_uint(acc[c + 6])), fin(__float_as_uint(acc[c + 7])));
-                o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
-                o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
-                *reinterpret_cast<uint4*>(y + c0 + c) = o;
-              }
-            } else {
-              if (XT) {
-                __half* yc = y + static_cast<long long>(c0) * a.ldy;
-#pragma unroll
-                for (int c = 0; c < 16; ++c, yc += a.ldy)
-                  if (c0 + c < a.N) *yc = __float2half_rn(fin(__float_as_uint(acc[c])));
+                for (int c = 0; c < CH; ++c)
+                  v[c] = __float_as_uint(__uint_as_float(v[c]) + __uint_as_float(lds_u32(p + static_cast<uint32_t>(c0 + c) * 512u)));
               } else {
+                const int c_id = c_first + 1 + k;
+                const int sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
+                const float* p = a.partials + static_cast<size_t>(sl) * NPAD * 128 + et;
 #pragma unroll
-                for (int c = 0; c < 16; ++c)
-                  if (c0 + c < a.N) y[c0 + c] = __float2half_rn(fin(__float_as_uint(acc[c])));
+                for (int c = 0; c < CH; ++c) v[c] = __float_as_uint(__uint_as_float(v[c]) + __ldcg(p + (c0 + c) * 128));
               }
             }
+            store_y(v, c0);
           }
         }
         tc_fence_before();
         mbar_arrive(bar_accempty + 8 * b);
-        if (et == 0) a.counters[mt] = 0;                          // leave the workspace cleared
-        named_bar_sync(1 + kGroups, 128);                         // last_flag is rewritten next segment
         TL3_TACC(2)
         ++seg;
         t = seg_end;
@@ -803,61 +826,9 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       tc_fence_before();
       mbar_arrive(bar_accempty + 8 * b);
       if (!complete) {
-        __threadfence();
+        __threadfence();                                          // the partial sums, before the flag
         named_bar_sync(1 + kGroups, 128);
-        if (et == 0) {
-          const unsigned int old = atomicAdd(a.counters + mt, 1u);
-          const bool last = old == static_cast<unsigned int>(c_last - c_first);
-          if (last) a.counters[mt] = 0;                          // leave the workspace cleared
-          *last_flag = last ? 1u : 0u;
-        }
-        named_bar_sync(1 + kGroups, 128);
-        if (*last_flag) {
-          __threadfence();
-          // The last segment of a CTA ends after all of its tiles: the stages are idle then, so the
-          // contributors' partial sums are fetched with one bulk copy each, all in flight at once,
-          // instead of one round trip of loads per contributor.
-          constexpr uint32_t kSlotBytes = NPAD * 128u * 4u;
-          const int n_contrib = c_last - c_first + 1;
-          const bool staged = seg_end == t_end && static_cast<uint32_t>(n_contrib) * kSlotBytes <= static_cast<uint32_t>(S) * a.stage_stride;
-          bool fetched = true;
-          if (staged) {
-            if (et == 0) {
-              fence_proxy_async_all();
-              mbar_arrive_expect_tx(bar_tail, static_cast<uint32_t>(n_contrib) * kSlotBytes);
-              for (int c_id = c_first, k = 0; c_id <= c_last; ++c_id, ++k) {
-                const int sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
-                bulk_copy_g2s(smem_base + static_cast<uint32_t>(k) * kSlotBytes, a.partials + static_cast<size_t>(sl) * NPAD * 128, kSlotBytes, bar_tail);
-              }
-            }
-            fetched = mbar_wait(bar_tail, 0, wctx, kStEpilogueTail);
-          }
-          if (fetched) {
-#pragma unroll 1
-            for (int c0 = 0; c0 < NPAD; c0 += CH) {
-              float acc[CH];
-#pragma unroll
-              for (int c = 0; c < CH; ++c) acc[c] = 0.f;
-              for (int c_id = c_first, k = 0; c_id <= c_last; ++c_id, ++k) {    // fixed order: deterministic sum
-                if (staged) {
-                  const uint32_t p = smem_base + (static_cast<uint32_t>(k) * NPAD * 128u + static_cast<uint32_t>(et)) * 4u;
-#pragma unroll
-                  for (int c = 0; c < CH; ++c) acc[c] += __uint_as_float(lds_u32(p + static_cast<uint32_t>(c0 + c) * 512u));
-                } else {
-                  const int sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
-                  const float* p = a.partials + static_cast<size_t>(sl) * NPAD * 128 + et;
-#pragma unroll
-                  for (int c = 0; c < CH; ++c) acc[c] += __ldcg(p + (c0 + c) * 128);
-                }
-              }
-              uint32_t v[CH];
-#pragma unroll
-              for (int c = 0; c < CH; ++c) v[c] = __float_as_uint(acc[c]);
-              store_y(v, c0);
-            }
-          }
-        }
-        named_bar_sync(1 + kGroups, 128);                         // last_flag may be rewritten next segment
+        if (et == 0) asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(a.flags + slot), "r"(1u) : "memory");
       }
       TL3_TACC(2)
       ++seg;
@@ -920,12 +891,13 @@ static EncodeTiledFn encode_tiled_fn() {
 static inline int n_pad_of(int N) { return N <= 16 ? 16 : N <= 32 ? 32 : 64; }
 
 struct WorkspaceLayout {
-  size_t status_off = 0, counters_off = 256, partials_off = 0, total = 0;
+  size_t status_off = 0, flags_off = 256, partials_off = 0, total = 0;
 };
 
 static WorkspaceLayout workspace_layout(const tl3_matrix* m, int n_pad, int sm_count) {
   WorkspaceLayout w;
-  w.partials_off = (256 + static_cast<size_t>(m->tiles_m) * 4 + 4095) / 4096 * 4096;
+  (void)m;
+  w.partials_off = (256 + static_cast<size_t>(2) * sm_count * 4 + 4095) / 4096 * 4096;
   w.total = w.partials_off + static_cast<size_t>(2) * sm_count * n_pad * 128 * sizeof(float);
   return w;
 }
@@ -1068,7 +1040,7 @@ static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, 
   args.bias = ep ? static_cast<const __half*>(ep->bias) : nullptr;
   args.act = ep ? ep->activation : TL3_ACT_NONE;
   args.partials = reinterpret_cast<float*>(ws + wl.partials_off);
-  args.counters = reinterpret_cast<unsigned int*>(ws + wl.counters_off);
+  args.flags = reinterpret_cast<unsigned int*>(ws + wl.flags_off);
   args.status = reinterpret_cast<unsigned int*>(ws + wl.status_off);
   args.stage_stride = stage_stride;
   args.x_offset = block_area;
@@ -1152,7 +1124,7 @@ int tl3_spmm_host(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int N, vo
 }
 
 // ---- entry point that allocates nothing: scratch inside the library image -------------------
-// Split-K partials, arrival counters and the status word for callers that cannot supply a
+// Split-K partials, their arrival flags and the status word for callers that cannot supply a
 // workspace.  The name below is a host-side handle of the symbol, not a device address: host code
 // must go through cudaGetSymbolAddress (done once per device, with that device current).
 static __device__ __align__(256) unsigned char g_static_scratch[TL3_STATIC_SCRATCH_BYTES];
@@ -1185,7 +1157,7 @@ int tl3_spmm_static_scratch(const tl3_matrix* m, const void* X, int64_t ldx, voi
   if (wl.total > TL3_STATIC_SCRATCH_BYTES) return TL3_ERR_SCRATCH_LIMIT;
   void* scratch = nullptr;
   if (int rc = tl3::static_scratch_address(&scratch)) return rc;
-  // counters and status word must start at zero; the partial-sum slots are always written before
+  // flags and status word must start at zero; the partial-sum slots are always written before
   // they are read, so the last call's contents there do not matter
   TL3_CUDA(cudaMemsetAsync(scratch, 0, wl.partials_off, static_cast<cudaStream_t>(stream)));
   return tl3_spmm(m, X, ldx, Y, ldy, N, scratch, stream);

@@ -21,7 +21,7 @@ def test_static_scratch_entry_point_matches_the_regular_one(oracle_mod):
     build.build_library()
     L = tl3.lib()
     # 8 row-tiles x 40 k-tiles: every row-tile is shared by many CTAs, so the scratch (partial
-    # sums, counters) is really used
+    # sums, arrival flags) is really used
     case = wl.Case(0, "static", 1024, 5120, 16, 321, 0.5, "magnitude")
     W, X = case.make_W(), case.make_X()
     m = tl3.encode(W)
