@@ -36,7 +36,7 @@ WORKLOAD = "config2_opt13b_shapes_50pct_N8_16_32"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch / its algorithmic bytes, from the
 # ncu capture summarised in profiles/tl3_spmm_kernel_8192x8192_n16.md (scaled by bytes, since
 # traffic grows in proportion to the blob)
-NCU_TRAFFIC_RATIO = 1.05
+NCU_TRAFFIC_RATIO = 1.03
 
 
 def log(*a):
