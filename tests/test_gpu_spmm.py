@@ -178,6 +178,28 @@ def test_fewer_stages_than_decode_groups(tl3, oracle_mod):
     check(oracle_mod, D, X, Y)
 
 
+def test_workspace_is_left_cleared_and_can_serve_another_matrix(tl3, oracle_mod):
+    """The split-K hand-over keeps one flag per partial-sum slot in the workspace and relies on
+    finding them all at zero: after a launch the head of the workspace (status word and flags)
+    must read zero again, and the same workspace must then serve a different matrix."""
+    import torch
+    a = wl.Case(0, "ws_a", 1024, 5120, 16, 501, 0.5, "magnitude")      # every row-tile shared by many CTAs
+    b = wl.Case(0, "ws_b", 2304, 1152, 16, 502, 0.5, "bernoulli")      # other tile counts, other sharing pattern
+    Wa, Xa, Wb, Xb = a.make_W(), a.make_X(), b.make_W(), b.make_X()
+    ma, mb = tl3.encode(Wa), tl3.encode(Wb)
+    ma.upload()
+    mb.upload()
+    n = max(ma.workspace_bytes(16), mb.workspace_bytes(16))
+    ws = torch.empty(n, dtype=torch.uint8, device="cuda")
+    assert tl3.lib().tl3_workspace_init(ws.data_ptr(), n, None) == tl3.OK
+    for m, W, X in ((ma, Wa, Xa), (mb, Wb, Xb), (ma, Wa, Xa)):
+        Y = m.spmm(device_X(X), workspace=ws)
+        torch.cuda.synchronize()
+        assert m.status(ws) == tl3.OK
+        assert int(ws[:4096].to(torch.int32).sum().item()) == 0
+        check(oracle_mod, W, X, Y.cpu().numpy(), with_oracle_spmm=False)
+
+
 def test_thousands_of_back_to_back_launches(tl3):
     """Five different launches in one CUDA graph, replayed without host synchronisation: every
     replay must leave the status words clear and reproduce the first result bit for bit (the
