@@ -429,22 +429,23 @@ def _time_graph(fn, reps=20):
 
 
 def run_sweep(args):
-    """Extra measurements beside the headline: `--sweep n|sparsity|stack`.  One JSON line per point.
+    """Extra measurements beside the headline: `--sweep n|sparsity|stack|large`.  One JSON line per point.
     Every matrix is uploaded in enough copies that a copy is evicted from L2 before it is used again."""
     import torch
     from paper_2607_08786_b200 import build, tl3
     build.build_library()
     peak, _ = measured_peak_gbs()
 
-    def point(case, label):
+    def point(case, label, verify_rows=0):
         W = case.make_W()
         m0 = tl3.encode(W)
-        copies = max(2, int(np.ceil(3 * 126e6 / m0.device_bytes())))
+        # a matrix larger than three times L2 evicts itself: one copy is enough
+        copies = max(1 if m0.device_bytes() > 3 * 126e6 else 2, int(np.ceil(3 * 126e6 / m0.device_bytes())))
         copies = min(copies, 12)
         ms = [m0] + [tl3.encode(W) for _ in range(copies - 1)]
         for m in ms:
             m.upload()
-        dense = [torch.from_numpy(W).cuda() for _ in range(min(copies, max(2, int(np.ceil(3 * 126e6 / W.nbytes)))))]
+        dense = [torch.from_numpy(W).cuda() for _ in range(min(copies, max(1 if W.nbytes > 3 * 126e6 else 2, int(np.ceil(3 * 126e6 / W.nbytes)))))]
         Xd = torch.from_numpy(case.make_X()).cuda()
         ws = m0.new_workspace(case.N)
         Y = torch.empty((case.M, case.N), dtype=torch.float16, device="cuda")
@@ -462,7 +463,17 @@ def run_sweep(args):
         assert m0.status(ws) == tl3.OK
         nbytes = m0.device_bytes() + case.K * case.N * 2 + case.M * case.N * 2
         st = m0.stats()
-        print(json.dumps({"sweep": args.sweep, "point": label, "M": case.M, "K": case.K, "N": case.N,
+        extra = {}
+        if verify_rows:
+            # sampled rows of Y against the plain definition in float64, tolerance of the benchmark spec
+            rows = np.random.default_rng(case.seed).choice(case.M, size=verify_rows, replace=False)
+            Xh = Xd.cpu().numpy().astype(np.float64)
+            Wr = W[rows].astype(np.float64)
+            ref, bound = Wr @ Xh, np.abs(Wr) @ np.abs(Xh)
+            err = np.abs(Y[torch.from_numpy(rows).cuda()].cpu().numpy().astype(np.float64) - ref)
+            extra["verified_rows"] = int(verify_rows)
+            extra["max_err_over_tol"] = round(float(np.max(err / (2e-3 * bound + 1e-3))), 4)
+        print(json.dumps({**extra, "sweep": args.sweep, "point": label, "M": case.M, "K": case.K, "N": case.N,
                           "sparsity": case.sparsity, "us": round(us, 2), "gbs": round(nbytes / us / 1e3, 1),
                           "frac_measured": round(nbytes / us / 1e3 / peak, 4),
                           "dense_equiv_tflops": round(2.0 * case.M * case.K * case.N / us / 1e6, 2),
@@ -477,6 +488,9 @@ def run_sweep(args):
     if args.sweep == "n":
         for N in (8, 16, 32, 64, 128, 256, 512):
             point(wl.Case(4, "n_sweep", 9216, 9216, N, 4000, 0.5, "row_scaled"), f"N={N}")
+    elif args.sweep == "large":
+        # the shape of the comparison against cuBLAS in the Introduction (its first figure: M/K/N = 66K/16K/32)
+        point(wl.Case(0, "paper_66k_16k_n32", 65536, 16384, 32, 6000, 0.5, "magnitude"), "65536x16384_n32", verify_rows=64)
     elif args.sweep == "sparsity":
         for case in wl.config_cases(3):
             point(case, case.name)
@@ -520,7 +534,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--single", type=int, nargs=3, metavar=("M", "K", "N"), help="run a few launches of one shape and exit")
     ap.add_argument("--launches", type=int, default=3)
-    ap.add_argument("--sweep", choices=["n", "sparsity", "stack"], help="extra measurements; one JSON line per point")
+    ap.add_argument("--sweep", choices=["n", "sparsity", "stack", "large"], help="extra measurements; one JSON line per point")
     ap.add_argument("--sparsity", type=float, default=0.5)
     args = ap.parse_args()
     if args.single:
