@@ -296,9 +296,16 @@ def run_ours(args, rank, local_rank, world):
         dY = torch.empty(c.M * c.N * 2, dtype=torch.uint8, device=dev)
         e2e_bufs.append((Xp.numpy(), Yp.numpy(), dX, dY))
 
+    # the nine products are independent: each is enqueued (copy in, kernel, copy out) on one of three
+    # streams in turn, so the copies of one overlap the kernel of another, and the step ends when all
+    # three streams have drained
+    e2e_streams = [torch.cuda.Stream(device=dev) for _ in range(3)]
+
     def step_e2e():
-        for L, (Xp, Yp, dX, dY) in zip(launches, e2e_bufs):
-            L["m"].spmm_host(Xp, Yp, dX, dY, L["ws"])
+        for i, (L, (Xp, Yp, dX, dY)) in enumerate(zip(launches, e2e_bufs)):
+            L["m"].spmm_host_async(Xp, Yp, dX, dY, L["ws"], stream=e2e_streams[i % 3])
+        for s in e2e_streams:
+            s.synchronize()
 
     for _ in range(3):
         step_e2e()

@@ -170,6 +170,13 @@ int tl3_spmm_nt(const tl3_matrix* m, const void* Xt, int64_t ldxt, void* Yt, int
 int tl3_spmm_host(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int N, void* dX, void* dY,
                   void* workspace, void* stream);
 
+/* The same without the wait: the three steps are only enqueued on `stream`.  X must stay valid and
+ * Y is defined once the stream has passed this point (cudaStreamSynchronize, an event).  Calls on
+ * different streams may be in flight together as long as each has its own dX, dY and workspace:
+ * the copies of one then overlap the kernel of another. */
+int tl3_spmm_host_async(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int N, void* dX, void* dY,
+                        void* workspace, void* stream);
+
 /* (No counterpart in the paper.)  Y = W X exactly as tl3_spmm computes it, for callers that are
  * not allowed to obtain device memory themselves and so cannot provide a workspace: a driver-level
  * plug-in whose host application hands it only the input and output buffers and forbids allocation

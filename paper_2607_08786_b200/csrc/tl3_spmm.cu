@@ -1109,17 +1109,26 @@ int tl3_spmm_nt(const tl3_matrix* m, const void* Xt, int64_t ldxt, void* Yt, int
   return TL3_OK;
 }
 
-int tl3_spmm_host(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int N, void* dX, void* dY, void* workspace, void* stream) {
+int tl3_spmm_host_async(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int N, void* dX, void* dY, void* workspace, void* stream) {
   if (!m || !X || !Y || !dX || !dY) return TL3_ERR_INVALID_ARG;
   if (N < 1 || N > TL3_MAX_N) return TL3_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // device copy of X with a leading dimension that satisfies the 16-byte rule
   const int64_t ldx = (N + 7) / 8 * 8;
-  TL3_CUDA(cudaMemcpy2DAsync(dX, static_cast<size_t>(ldx) * 2, X, static_cast<size_t>(N) * 2, static_cast<size_t>(N) * 2,
-                             static_cast<size_t>(m->K), cudaMemcpyHostToDevice, st));
+  if (ldx == N) {
+    TL3_CUDA(cudaMemcpyAsync(dX, X, static_cast<size_t>(m->K) * N * 2, cudaMemcpyHostToDevice, st));
+  } else {
+    TL3_CUDA(cudaMemcpy2DAsync(dX, static_cast<size_t>(ldx) * 2, X, static_cast<size_t>(N) * 2, static_cast<size_t>(N) * 2,
+                               static_cast<size_t>(m->K), cudaMemcpyHostToDevice, st));
+  }
   if (int rc = tl3_spmm(m, dX, ldx, dY, N, N, workspace, stream)) return rc;
   TL3_CUDA(cudaMemcpyAsync(Y, dY, static_cast<size_t>(m->M) * N * 2, cudaMemcpyDeviceToHost, st));
-  TL3_CUDA(cudaStreamSynchronize(st));
+  return TL3_OK;
+}
+
+int tl3_spmm_host(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int N, void* dX, void* dY, void* workspace, void* stream) {
+  if (int rc = tl3_spmm_host_async(m, X, Y, N, dX, dY, workspace, stream)) return rc;
+  TL3_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
   return TL3_OK;
 }
 

@@ -27,7 +27,7 @@ _CANONICAL_DTYPES = (np.uint16, np.uint8, np.uint16, np.uint16, np.uint8, np.uin
 # every symbol include/tl3.h declares
 SYMBOLS = ("tl3_encode", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_deserialize",
            "tl3_free", "tl3_device_bytes", "tl3_pack", "tl3_upload", "tl3_workspace_bytes", "tl3_workspace_init",
-           "tl3_spmm", "tl3_spmm_ex", "tl3_spmm_nt", "tl3_spmm_host", "tl3_spmm_static_scratch", "tl3_static_scratch_status", "tl3_status", "tl3_status_word", "tl3_last_launch", "tl3_strerror",
+           "tl3_spmm", "tl3_spmm_ex", "tl3_spmm_nt", "tl3_spmm_host", "tl3_spmm_host_async", "tl3_spmm_static_scratch", "tl3_static_scratch_status", "tl3_status", "tl3_status_word", "tl3_last_launch", "tl3_strerror",
            "tl3_last_cuda_error")
 
 
@@ -91,6 +91,7 @@ def lib() -> ctypes.CDLL:
         L.tl3_spmm_ex.argtypes = [vp, vp, i64, vp, i64, ci, ctypes.POINTER(Epilogue), vp, vp]
         L.tl3_spmm_nt.argtypes = [vp, vp, i64, vp, i64, ci, ctypes.POINTER(Epilogue), vp, vp]
         L.tl3_spmm_host.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp]
+        L.tl3_spmm_host_async.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp]
         L.tl3_spmm_static_scratch.argtypes = [vp, vp, i64, vp, i64, ci, vp]
         L.tl3_static_scratch_status.argtypes = [vp]
         L.tl3_status.argtypes = [vp, vp, vp]
@@ -309,6 +310,15 @@ class Matrix:
             raise TypeError("Y must be a contiguous fp16/uint16 array")
         _check(lib().tl3_spmm_host(self._h, X.ctypes.data, Y.ctypes.data, X.shape[1], dX.data_ptr(),
                                    dY.data_ptr(), workspace.data_ptr(), _stream_ptr(stream)), "tl3_spmm_host")
+
+    def spmm_host_async(self, X: np.ndarray, Y: np.ndarray, dX, dY, workspace, stream=None) -> None:
+        """As :meth:`spmm_host` but only enqueued on ``stream``: ``X`` must stay alive and ``Y`` is
+        defined once the stream has been synchronised."""
+        X = _u16(X)
+        if Y.dtype not in (np.uint16, np.float16) or not Y.flags.c_contiguous:
+            raise TypeError("Y must be a contiguous fp16/uint16 array")
+        _check(lib().tl3_spmm_host_async(self._h, X.ctypes.data, Y.ctypes.data, X.shape[1], dX.data_ptr(),
+                                         dY.data_ptr(), workspace.data_ptr(), _stream_ptr(stream)), "tl3_spmm_host_async")
 
     def status(self, workspace, stream=None) -> int:
         return int(lib().tl3_status(self._h, workspace.data_ptr(), _stream_ptr(stream)))

@@ -371,6 +371,37 @@ def test_host_buffer_entry_point(tl3, oracle_mod):
     check(oracle_mod, W, X, Y)
 
 
+def test_host_buffer_entry_point_async_on_several_streams(tl3, oracle_mod):
+    """Three products enqueued on three streams (own staging buffers and workspaces), one wait at
+    the end: each result equals what the blocking call gives."""
+    import torch
+    cases = [wl.Case(0, "ha", 1024, 2560, 16, 21, 0.5, "magnitude"), wl.Case(0, "hb", 2560, 1024, 8, 22, 0.5, "magnitude"),
+             wl.Case(0, "hc", 640, 512, 12, 23, 0.5, "bernoulli")]
+    streams = [torch.cuda.Stream() for _ in cases]
+    jobs = []
+    for c in cases:
+        W, X = c.make_W(), c.make_X()
+        m = tl3.encode(W)
+        m.upload()
+        Xp = torch.from_numpy(X).pin_memory()
+        Yp = torch.zeros((c.M, c.N), dtype=torch.float16).pin_memory()
+        dX = torch.empty(c.K * ((c.N + 7) // 8 * 8) * 2, dtype=torch.uint8, device="cuda")
+        dY = torch.empty(c.M * c.N * 2, dtype=torch.uint8, device="cuda")
+        jobs.append((c, W, X, m, Xp, Yp, dX, dY, m.new_workspace(c.N)))
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for (c, W, X, m, Xp, Yp, dX, dY, ws), st in zip(jobs, streams):
+            m.spmm_host_async(Xp.numpy(), Yp.numpy(), dX, dY, ws, stream=st)
+    for st in streams:
+        st.synchronize()
+    for c, W, X, m, Xp, Yp, dX, dY, ws in jobs:
+        assert m.status(ws) == tl3.OK
+        check(oracle_mod, W, X, Yp.numpy(), with_oracle_spmm=False)
+        Yb = np.zeros((c.M, c.N), dtype=np.float16)
+        m.spmm_host(X, Yb, dX, dY, ws)
+        assert np.array_equal(Yb.view(np.uint16), Yp.numpy().view(np.uint16))
+
+
 def _sampled_check(oracle_mod, W, X, Y, rows):
     Yref, bound = oracle_mod.dense_fp64(W[rows], X)
     err = np.abs(Y[rows].astype(np.float64) - Yref)
