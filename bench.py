@@ -37,6 +37,8 @@ WORKLOAD = "config2_opt13b_shapes_50pct_N8_16_32"
 # ncu capture summarised in profiles/tl3_spmm_kernel_8192x8192_n16.md (scaled by bytes, since
 # traffic grows in proportion to the blob)
 NCU_TRAFFIC_RATIO = 1.03
+# streams the independent products of a step are forked over inside the graph
+N_STREAMS = 3
 
 
 def log(*a):
@@ -186,15 +188,56 @@ def run_ours(args, rank, local_rank, world):
         for L in launches:
             L["m"].spmm(L["X"], L["Y"], workspace=L["ws"])
 
-    # the nine launches as one CUDA graph (removes host launch gaps); eager if capture is refused
-    graph = None
-    try:
-        step_eager()
+    # The nine products of a step are independent of each other (own X, Y, workspace).  In the
+    # graph they are forked over N_STREAMS streams (launch i on stream i % N_STREAMS, joined at the
+    # end of the step), which tells CUDA as much: a kernel then takes over SMs as the CTAs of a
+    # kernel on another stream leave, instead of waiting for that whole grid as the next kernel on
+    # the same stream must.  The dense baseline is captured the same way.
+    side_streams = [torch.cuda.Stream(device=dev) for _ in range(N_STREAMS - 1)]
+
+    def forked(calls):
+        def run():
+            cur = torch.cuda.current_stream()
+            ev = torch.cuda.Event()
+            ev.record(cur)
+            for s in side_streams:
+                s.wait_event(ev)
+            for i, call in enumerate(calls):
+                st = cur if i % N_STREAMS == 0 else side_streams[i % N_STREAMS - 1]
+                with torch.cuda.stream(st):
+                    call()
+            for s in side_streams:
+                done = torch.cuda.Event()
+                done.record(s)
+                cur.wait_event(done)
+        return run
+
+    def capture(fn):
+        fn()
         torch.cuda.synchronize()
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
-            step_eager()
-        graph = g
+            fn()
+        return g
+
+    def time_replays(g, n):
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(torch.cuda.current_stream())
+        for _ in range(n):
+            g.replay()
+        b.record(torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    spmm_calls = [(lambda L=L: L["m"].spmm(L["X"], L["Y"], workspace=L["ws"])) for L in launches]
+    # the step as one CUDA graph (removes host launch gaps); eager on one stream if capture is refused
+    graph, serial_ms = None, None
+    try:
+        graph = capture(forked(spmm_calls))
+        serial_ms = time_replays(capture(step_eager), max(10, min(args.steps, 100)))   # all nine on one stream, for reference
     except Exception as e:  # pragma: no cover
         log(f"[rank {rank}] CUDA graph capture failed ({e}); timing eager launches")
         graph = None
@@ -255,22 +298,12 @@ def run_ours(args, rank, local_rank, world):
 
     dense_step()
     torch.cuda.synchronize()
-    dense_graph_ms = None
+    dense_graph_ms, dense_serial_ms = None, None
     try:
-        dg = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(dg):
-            dense_step()
-        for _ in range(3):
-            dg.replay()
-        torch.cuda.synchronize()
-        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        dense_calls = [(lambda i=i, L=L: torch.matmul(dense[(L["case"].M, L["case"].K)], L["X"], out=outs[i])) for i, L in enumerate(launches)]
         nrep = max(10, min(args.steps, 100))
-        d0.record(stream)
-        for _ in range(nrep):
-            dg.replay()
-        d1.record(stream)
-        torch.cuda.synchronize()
-        dense_graph_ms = d0.elapsed_time(d1) / nrep
+        dense_graph_ms = time_replays(capture(forked(dense_calls)), nrep)
+        dense_serial_ms = time_replays(capture(dense_step), nrep)
     except Exception as e:  # pragma: no cover
         log(f"[rank {rank}] dense graph capture failed ({e})")
     dper = [[] for _ in launches]
@@ -372,6 +405,7 @@ def run_ours(args, rank, local_rank, world):
         "config": {"workload": WORKLOAD, "launches_per_step": len(launches), "order": "N-major",
                    "l2": "inputs larger than L2: 297 MB of other weights stream between two uses of a matrix",
                    "bytes_per_step": step_bytes, "graph": graph is not None,
+                   "streams": N_STREAMS if graph is not None else 1,
                    "ctas": ll["ctas"], "smem_bytes": ll["smem_bytes"]},
         "clocks": clocks,
         "gpu_launches": len(launches) * args.steps,
@@ -383,6 +417,9 @@ def run_ours(args, rank, local_rank, world):
                      "kernel": "tl3_spmm_kernel", "avg_launch_us": ms_step * 1e3 / len(launches),
                      "algorithmic_bytes_per_launch": step_bytes / len(launches)},
         "cpu_baseline": cpu,
+        "single_stream": {"ms_per_step": serial_ms, "value": (step_bytes / (serial_ms * 1e-3) / 1e9) if serial_ms else None,
+                          "dense_ms_per_step": dense_serial_ms,
+                          "note": "the same nine launches as a graph on one stream: each kernel waits for the whole grid before it"},
         "dense_fp16_gemm": {"ms_per_step_graph": dense_graph_ms,
                             "speedup_of_spmm_graph": (dense_graph_ms / ms_step) if dense_graph_ms else None,
                             "us_per_step_eager": sum(dus), "spmm_us_per_step_eager": sum(us)},
