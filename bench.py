@@ -157,28 +157,32 @@ def run_ours(args, rank, local_rank, world):
     dev = torch.device("cuda", local_rank)
 
     cases = step_cases(dist.rank_seed_offset(rank))
-    mats, dense = {}, {}
+    # Every launch of a step reads its own device copy of its weight matrix (and the dense baseline
+    # its own dense copy), so no weight byte is touched twice within a step whatever order the
+    # concurrent kernels end up running in; a step streams 918 MB, seven times the L2.
+    host_W = {}
     launches = []
     t_setup = time.time()
     for c in cases:
         key = (c.M, c.K)
-        if key not in mats:
-            W = c.make_W()
-            m = tl3.encode(W)
-            m.upload(device=dev)
-            mats[key] = m
-            dense[key] = torch.from_numpy(W).to(dev)
+        first = key not in host_W
+        if first:
+            host_W[key] = c.make_W()
+        W = host_W[key]
+        m = tl3.encode(W)
+        m.upload(device=dev)
+        dW = torch.from_numpy(W).to(dev)
+        if first:
             st = m.stats()
             log(f"[rank {rank}] {c.M}x{c.K}: nnz {st['nnz']} TC {st['n_tc']/st['nnz']:.4f} SF {st['n_sf']/st['nnz']:.4f} "
                 f"RES {st['n_res']/st['nnz']:.4f} dummies {st['n_dummy']/st['nnz']:.4f} blob {st['device_bytes']/1e6:.1f} MB "
                 f"({st['device_bytes']/(2*c.M*c.K):.4f} x dense, canonical {st['canonical_bytes']/(2*c.M*c.K):.4f})")
-        m = mats[key]
         X = c.make_X()
         Xd = torch.from_numpy(X).to(dev)
         Y = torch.empty((c.M, c.N), dtype=torch.float16, device=dev)
         ws = m.new_workspace(c.N)
         nbytes = m.device_bytes() + X.nbytes + c.M * c.N * 2
-        launches.append(dict(case=c, m=m, X=Xd, Y=Y, ws=ws, bytes=nbytes, Xh=X, flops=2.0 * c.M * c.K * c.N))
+        launches.append(dict(case=c, m=m, X=Xd, Y=Y, ws=ws, bytes=nbytes, Xh=X, flops=2.0 * c.M * c.K * c.N, dense=dW))
     torch.cuda.synchronize()
     log(f"[rank {rank}] setup {time.time() - t_setup:.1f} s")
 
@@ -294,13 +298,13 @@ def run_ours(args, rank, local_rank, world):
 
     def dense_step():
         for i, L in enumerate(launches):
-            torch.matmul(dense[(L["case"].M, L["case"].K)], L["X"], out=outs[i])
+            torch.matmul(L["dense"], L["X"], out=outs[i])
 
     dense_step()
     torch.cuda.synchronize()
     dense_graph_ms, dense_serial_ms = None, None
     try:
-        dense_calls = [(lambda i=i, L=L: torch.matmul(dense[(L["case"].M, L["case"].K)], L["X"], out=outs[i])) for i, L in enumerate(launches)]
+        dense_calls = [(lambda i=i, L=L: torch.matmul(L["dense"], L["X"], out=outs[i])) for i, L in enumerate(launches)]
         nrep = max(10, min(args.steps, 100))
         dense_graph_ms = time_replays(capture(forked(dense_calls)), nrep)
         dense_serial_ms = time_replays(capture(dense_step), nrep)
@@ -311,7 +315,7 @@ def run_ours(args, rank, local_rank, world):
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(launches) + 1)]
         evs[0].record(stream)
         for i, L in enumerate(launches):
-            torch.matmul(dense[(L["case"].M, L["case"].K)], L["X"], out=outs[i])
+            torch.matmul(L["dense"], L["X"], out=outs[i])
             evs[i + 1].record(stream)
         torch.cuda.synchronize()
         if rep >= 2:
@@ -403,7 +407,7 @@ def run_ours(args, rank, local_rank, world):
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f16xf16->f32", "data": "synthetic",
         "config": {"workload": WORKLOAD, "launches_per_step": len(launches), "order": "N-major",
-                   "l2": "inputs larger than L2: 297 MB of other weights stream between two uses of a matrix",
+                   "l2": "inputs larger than L2: every launch of a step reads its own copy of W, a step streams 918 MB",
                    "bytes_per_step": step_bytes, "graph": graph is not None,
                    "streams": N_STREAMS if graph is not None else 1,
                    "ctas": ll["ctas"], "smem_bytes": ll["smem_bytes"]},
