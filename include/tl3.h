@@ -208,6 +208,14 @@ int tl3_static_scratch_status(void* stream);
 int tl3_status(const tl3_matrix* m, void* workspace, void* stream);
 int tl3_status_word(void* workspace, void* stream, uint32_t* word);
 
+/* Self-test of the kernels' bounded waits (every wait inside the kernels gives up after 2 s,
+ * records a code in the status word and lets the kernel return).  Enqueues a one-CTA kernel that
+ * waits on a barrier nothing ever arrives at; about 2 s after it starts, tl3_status() on the
+ * same workspace reports DEVICE_TIMEOUT (code 1), the second word of the workspace holds 2
+ * ("gave up"; 1 would mean the wait completed), and the device is usable as before.  Clear the
+ * workspace with tl3_workspace_init() before using it for a product again. */
+int tl3_selftest_bounded_wait(void* workspace, void* stream);
+
 /* Kernel launch geometry of the last tl3_spmm on this handle (for reporting): CTAs, stages. */
 int tl3_last_launch(const tl3_matrix* m, int* ctas, int* stages, int* smem_bytes);
 

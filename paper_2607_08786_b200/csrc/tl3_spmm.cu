@@ -846,6 +846,23 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   }
 }
 
+// Self-test of the bounded wait: one CTA waits on a barrier that nothing ever arrives at.  The
+// wait gives up after its limit, records its code in the status word and the kernel returns; the
+// context stays usable.
+__global__ void bounded_wait_probe_kernel(unsigned int* status, unsigned int* outcome) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const WaitCtx w{&abort_flag, status, global_timer()};
+  const bool completed = mbar_wait(smem_u32(&bar), 0, w, kStProducer);
+  if (threadIdx.x == 0) *outcome = completed ? 1u : 2u;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
@@ -1204,6 +1221,14 @@ int tl3_last_launch(const tl3_matrix* m, int* ctas, int* stages, int* smem_bytes
 }
 
 int tl3_last_cuda_error(void) { return tl3::g_last_cuda_error; }
+
+int tl3_selftest_bounded_wait(void* workspace, void* stream) {
+  if (!workspace) return TL3_ERR_INVALID_ARG;
+  unsigned int* words = static_cast<unsigned int*>(workspace);
+  tl3::bounded_wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(words, words + 1);
+  TL3_CUDA(cudaGetLastError());
+  return TL3_OK;
+}
 
 #ifdef TL3_PHASE_TIMING
 void tl3_debug_set_timing_buffer(long long* device_ptr) { tl3::g_timing_buffer = device_ptr; }

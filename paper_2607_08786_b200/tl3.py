@@ -27,7 +27,7 @@ _CANONICAL_DTYPES = (np.uint16, np.uint8, np.uint16, np.uint16, np.uint8, np.uin
 # every symbol include/tl3.h declares
 SYMBOLS = ("tl3_encode", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_deserialize",
            "tl3_free", "tl3_device_bytes", "tl3_pack", "tl3_upload", "tl3_workspace_bytes", "tl3_workspace_init",
-           "tl3_spmm", "tl3_spmm_ex", "tl3_spmm_nt", "tl3_spmm_host", "tl3_spmm_host_async", "tl3_spmm_static_scratch", "tl3_static_scratch_status", "tl3_status", "tl3_status_word", "tl3_last_launch", "tl3_strerror",
+           "tl3_spmm", "tl3_spmm_ex", "tl3_spmm_nt", "tl3_spmm_host", "tl3_spmm_host_async", "tl3_spmm_static_scratch", "tl3_static_scratch_status", "tl3_status", "tl3_status_word", "tl3_selftest_bounded_wait", "tl3_last_launch", "tl3_strerror",
            "tl3_last_cuda_error")
 
 
@@ -96,6 +96,7 @@ def lib() -> ctypes.CDLL:
         L.tl3_static_scratch_status.argtypes = [vp]
         L.tl3_status.argtypes = [vp, vp, vp]
         L.tl3_status_word.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+        L.tl3_selftest_bounded_wait.argtypes = [vp, vp]
         L.tl3_last_launch.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci)]
         L.tl3_strerror.argtypes = [ci]
         L.tl3_strerror.restype = ctypes.c_char_p

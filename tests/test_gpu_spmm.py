@@ -357,6 +357,31 @@ def test_argument_errors_on_device(tl3):
     assert m.status(ws) == tl3.OK
 
 
+def test_a_wait_that_nothing_ends_gives_up_and_reports(tl3, oracle_mod):
+    """Every wait inside the kernels is bounded.  The library's self-test waits on a barrier that
+    nothing arrives at: the kernel must return by itself, the status must say which wait gave up,
+    and the device must work as before."""
+    import time
+    import torch
+    case = wl.Case(0, "after_timeout", 512, 1024, 8, 31, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    m = tl3.encode(W)
+    m.upload()
+    ws = m.new_workspace(case.N)
+    stream = torch.cuda.current_stream().cuda_stream
+    t0 = time.time()
+    assert tl3.lib().tl3_selftest_bounded_wait(ws.data_ptr(), stream) == tl3.OK
+    assert m.status(ws) == tl3.ERR_DEVICE_TIMEOUT          # synchronises: returns when the kernel has given up
+    assert 1.0 < time.time() - t0 < 30.0
+    assert m.status_word(ws) & 0xFF == 1
+    assert int(ws[4:8].view(torch.int32).item()) == 2      # the wait gave up, it did not complete
+    assert tl3.lib().tl3_workspace_init(ws.data_ptr(), ws.numel(), stream) == tl3.OK
+    Y = m.spmm(device_X(X), workspace=ws)
+    torch.cuda.synchronize()
+    assert m.status(ws) == tl3.OK
+    check(oracle_mod, W, X, Y.cpu().numpy(), with_oracle_spmm=False)
+
+
 def test_host_buffer_entry_point(tl3, oracle_mod):
     import torch
     case = wl.Case(0, "h", 640, 512, 12, 8, 0.5, "magnitude")
