@@ -357,6 +357,28 @@ def test_argument_errors_on_device(tl3):
     assert m.status(ws) == tl3.OK
 
 
+def test_random_shapes_widths_and_masks(tl3, oracle_mod):
+    """Forty seeded random problems: ragged M and K, every width from 1 to 80, sparsities 30-90 %,
+    all four mask kinds, wide-and-flat and tall-and-thin matrices (many or no CTAs per row-tile).
+    Each one twice: within tolerance of the float64 definition, same bits both times, status clear."""
+    import torch
+    rng = np.random.default_rng(20260)
+    for _ in range(40):
+        M = int(rng.integers(1, 24)) * 128 + int(rng.choice([0, 0, 0, 1, 37, 64, 127]))
+        K = int(rng.integers(1, 24)) * 128 + int(rng.choice([0, 0, 0, 8, 40, 120]))
+        if rng.random() < 0.25:
+            a, b = int(rng.integers(1, 4)) * 128, int(rng.integers(40, 120)) * 128
+            M, K = (a, b) if rng.random() < 0.5 else (b, a)
+        N = int(rng.choice([1, 3, 8, 12, 16, 24, 32, 48, 64, 80]))
+        case = wl.Case(0, "rnd", M, K, N, int(rng.integers(0, 1 << 30)), float(rng.choice([0.3, 0.4, 0.5, 0.5, 0.6, 0.7, 0.9])),
+                       str(rng.choice(["magnitude", "bernoulli", "row_scaled", "wanda"])))
+        W, X = case.make_W(), case.make_X()
+        Y, m = run_gpu(tl3, W, X, repeats=2)
+        check(oracle_mod, W, X, Y, with_oracle_spmm=False)
+        m.close()
+        torch.cuda.empty_cache()
+
+
 def test_a_wait_that_nothing_ends_gives_up_and_reports(tl3, oracle_mod):
     """Every wait inside the kernels is bounded.  The library's self-test waits on a barrier that
     nothing arrives at: the kernel must return by itself, the status must say which wait gave up,
