@@ -539,6 +539,8 @@ def run_sweep(args):
     elif args.sweep == "large":
         # the shape of the comparison against cuBLAS in the Introduction (its first figure: M/K/N = 66K/16K/32)
         point(wl.Case(0, "paper_66k_16k_n32", 65536, 16384, 32, 6000, 0.5, "magnitude"), "65536x16384_n32", verify_rows=64)
+        # the same matrix at N = 16, where a stage is small enough for the kernel to run six of them
+        point(wl.Case(0, "paper_66k_16k_n16", 65536, 16384, 16, 6000, 0.5, "magnitude"), "65536x16384_n16", verify_rows=64)
     elif args.sweep == "sparsity":
         for case in wl.config_cases(3):
             point(case, case.name)
