@@ -733,6 +733,10 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         // the stages, idle by now), so that when the last contributor arrives only its slot is
         // still to come.  The sum runs in ascending CTA order whatever the order of arrival: the
         // result does not depend on timing.
+        // Progress: a contributor waits for nobody, so it finishes once it holds an SM; the reducer
+        // waits only for CTAs with a higher index, and blocks are dispatched in index order, so only
+        // the reducers just below a launch's dispatch front can be waiting for a CTA that is not
+        // resident yet.  The wait is bounded all the same (status code kStEpilogueFlags).
         constexpr uint32_t kSlotBytes = NPAD * 128u * 4u;
         const bool staged = seg_end == t_end && static_cast<uint32_t>(n_others) * kSlotBytes <= static_cast<uint32_t>(S) * a.stage_stride;
         bool ok = true;
