@@ -235,6 +235,54 @@ def test_thousands_of_back_to_back_launches(tl3):
             assert torch.equal(Y, ref), c.name
 
 
+def test_concurrent_launches_on_several_streams(tl3):
+    """The same five launches forked over three streams inside one CUDA graph, so that kernels of
+    different streams share the GPU (a kernel moves in as another moves out, and CTAs of a launch
+    may still be waiting for an SM while its reducers already collect): results and status as in
+    the serial run, replay after replay."""
+    import torch
+    cases = [wl.Case(0, "a", 2560, 5120, 16, 1, 0.5, "magnitude"), wl.Case(0, "b", 2048, 8192, 32, 2, 0.5, "magnitude"),
+             wl.Case(0, "c", 2048, 2048, 64, 3, 0.4, "magnitude"), wl.Case(0, "d", 1024, 1024, 8, 4, 0.5, "bernoulli"),
+             wl.Case(0, "e", 3000, 3000, 24, 5, 0.7, "magnitude")]
+    L = []
+    for c in cases:
+        m = tl3.encode(c.make_W())
+        m.upload()
+        Xd = device_X(c.make_X())
+        ws = m.new_workspace(c.N)
+        Y = torch.empty((c.M, c.N), dtype=torch.float16, device="cuda")
+        m.spmm(Xd, Y, workspace=ws)
+        torch.cuda.synchronize()
+        L.append((c, m, Xd, Y, ws, Y.clone()))
+    side = [torch.cuda.Stream() for _ in range(2)]
+
+    def step():
+        cur = torch.cuda.current_stream()
+        start = torch.cuda.Event()
+        start.record(cur)
+        for s in side:
+            s.wait_event(start)
+        for i, (c, m, Xd, Y, ws, ref) in enumerate(L):
+            m.spmm(Xd, Y, workspace=ws, stream=cur if i % 3 == 0 else side[i % 3 - 1])
+        for s in side:
+            done = torch.cuda.Event()
+            done.record(s)
+            cur.wait_event(done)
+
+    step()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    for _ in range(5):
+        for _ in range(100):
+            g.replay()
+        torch.cuda.synchronize()
+        for c, m, Xd, Y, ws, ref in L:
+            assert m.status_word(ws) == 0, c.name
+            assert torch.equal(Y, ref), c.name
+
+
 def test_identity_X_reproduces_W_bit_for_bit(tl3):
     """Each y_ij is one product w_ij * 1: the GPU must hand back the decoded W exactly."""
     for k0 in (0, 64):
