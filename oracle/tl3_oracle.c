@@ -20,10 +20,10 @@
  *   tc_vals  u16[M_pad][K_pad/2]   two value slots per window of four consecutive weights
  *   tc_meta  u8 [M_pad][K_pad/8]   one nibble per window: idx0 | idx1<<2 (2 bits per value,
  *                                  Sec. 3.2 Sparse-TC layer), even window in the low nibble
- *   chain_tau0, chain_rho0 u16[tiles][TM]   16-bit first positions of Algorithm 1 (lines 3-4)
+ *   chain_tau0, chain_rho0 u16[tiles][TM]   16-bit first positions of Algorithm 1 (its initial offsets)
  *   chain_len u8[tiles][TM]        number of delta bytes of the chain (replaces BitLen(code))
  *   pdd_bytes u8[]                 delta bytes, low nibble = offset_t delta, high nibble =
- *                                  offset_r delta (Algorithm 1 lines 8-9); a zero nibble marks a
+ *                                  offset_r delta (Algorithm 1, the two 4-bit advances); a zero nibble marks a
  *                                  dummy point (Sec. 3.2: spans above the 4-bit range are broken up)
  *   tile_dir u32[tiles][4]         {pdd_off, pdd_len, res_off, res_cnt}
  *   res_rho u16[], res_val u16[]   Residual layer: (position, value) per tile [Sec. 3.2]
