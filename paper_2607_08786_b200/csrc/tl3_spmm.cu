@@ -329,8 +329,8 @@ __device__ __forceinline__ void decode_chain(uint32_t stage, uint32_t wr, uint32
     const uint32_t off2 = swizzled_offset2(pos);
     const uint32_t at = stage + (off2 & 0xFFFFu);
     const uint32_t v = lds_u16(at);
-    sts_u16(at, 0);                                     // W_t[offset_t] = 0
-    sts_u16(wr + (off2 >> 16), v);                      // W_r[offset_r] = W_t[offset_t]
+    sts_u16(at, 0);                                     // the slot it was parked in is empty again
+    sts_u16(wr + (off2 >> 16), v);                      // the value goes to its own position in W_r
   }
 #pragma unroll
   for (int k = 0; k < 3; ++k) {                         // one code word = four delta bytes
