@@ -136,7 +136,14 @@ int tl3_workspace_init(void* workspace, size_t bytes, void* stream);
  *   again.  fp32 accumulation, fp16 round-to-nearest-even output.  W and X are assumed finite (an
  *   empty slot multiplies an exact zero with an element of X).
  * Asynchronous on `stream`; allocates nothing; does not synchronise.  Calls that share a
- * workspace must not overlap on the GPU.
+ * workspace must not overlap on the GPU; the workspace must hold tl3_workspace_bytes(m, N) bytes
+ * for THIS N (it grows with N: 16, 32 or 64 columns of partial sums per slot), the call cannot
+ * check that.  Calls on different streams, each with its own workspace, may be in flight together.
+ * A row-tile shared by several CTAs is finished by the CTA that owns its first tile, which waits
+ * (bounded, status code 11) for CTAs with a higher index; that those get to run while other
+ * kernels hold SMs rests on the GPU dispatching the blocks of a grid in index order.
+ * Threads: calls that take a const handle may share it; tl3_upload() and tl3_free() may not run
+ * beside another call on the same handle.
  * Errors: NOT_UPLOADED, INVALID_ARG, UNSUPPORTED (N out of range, device is not sm_100), CUDA. */
 #define TL3_MAX_N 4096
 int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N,
@@ -184,13 +191,15 @@ int tl3_spmm_host_async(const tl3_matrix* m, const uint16_t* X, uint16_t* Y, int
  * spent before this library was loaded.  The split-K partial sums, the arrival flags and the
  * status word live in a fixed array that is part of the library image: TL3_STATIC_SCRATCH_BYTES
  * (3 MiB) of device memory on every GPU that loads the library, held until the process exits.
- *   - Problems whose scratch need (what tl3_workspace_bytes() reports) exceeds that size are refused
- *     with TL3_ERR_SCRATCH_LIMIT and nothing is launched.  On a 148-SM device this admits N <= 16
- *     for any matrix with up to ~150000 row-tiles; N > 16 is refused there.
+ *   - Problems whose scratch need (what tl3_workspace_bytes() reports; it depends on the SM count
+ *     and on N, not on the matrix) exceeds that size are refused with TL3_ERR_SCRATCH_LIMIT and
+ *     nothing is launched.  On a 148-SM device this admits N <= 16; N > 16 is refused there.
  *   - X, Y, ldx, ldy, N, stream: as for tl3_spmm.  The caller still owns X and Y.
  *   - The first call on each device looks up the array's device address (that device must be
  *     current); make that first call outside any stream capture.  Later calls only enqueue work.
- *   - The function calls no cudaMalloc / cudaFree nor any allocating routine, on any call.
+ *   - No call obtains device memory: no cudaMalloc / cudaFree, no allocating library routine.
+ *     The first call per device does one-time host-side set-up (the address look-up, the kernel's
+ *     shared-memory opt-in, the driver's lazy loading of the kernel image).
  *   - All calls on a device share the one array.  Each call clears the flags and the status word
  *     on `stream` before the kernel, so a call that was cut short does not poison the next one, but
  *     two calls that overlap on the GPU (different streams, no dependency) race on it: serialise
@@ -215,6 +224,20 @@ int tl3_status_word(void* workspace, void* stream, uint32_t* word);
  * ("gave up"; 1 would mean the wait completed), and the device is usable as before.  Clear the
  * workspace with tl3_workspace_init() before using it for a product again. */
 int tl3_selftest_bounded_wait(void* workspace, void* stream);
+
+/* (No counterpart in the paper.)  Launch tuning, process-wide, read by every later tl3_spmm* call.
+ *   decode_before_x  launches with at most this many tiles per CTA decode a block as soon as it is
+ *                    in shared memory instead of waiting for its X tile as well (X may come from the
+ *                    kernel before, which the launch overlaps; the weights never do).  Measured on
+ *                    B200: 9 % faster at one tile per CTA (1024 x 1024), level or up to 1 % slower
+ *                    from seven tiles per CTA on.  0 = never, -1 = always.
+ * tl3_set_tuning(NULL) restores the default.  Errors: INVALID_ARG. */
+#define TL3_DEFAULT_DECODE_BEFORE_X 4
+typedef struct {
+  int32_t decode_before_x;
+} tl3_tuning;
+int tl3_get_tuning(tl3_tuning* out);
+int tl3_set_tuning(const tl3_tuning* t);
 
 /* Kernel launch geometry of the last tl3_spmm on this handle (for reporting): CTAs, stages. */
 int tl3_last_launch(const tl3_matrix* m, int* ctas, int* stages, int* smem_bytes);

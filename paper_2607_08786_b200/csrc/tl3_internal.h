@@ -1,7 +1,9 @@
 // Internal definitions shared by the host-side and CUDA-side translation units of libtl3.
 #pragma once
+#include <atomic>
 #include <cstdint>
 #include <cstddef>
+#include <mutex>
 #include <vector>
 
 #include "tl3.h"
@@ -25,13 +27,18 @@ struct tl3_matrix {
 
   // device binding (filled by tl3_upload)
   void* dptr = nullptr;
-  size_t device_bytes = 0;             // computed lazily by tl3_device_bytes
-  uint32_t max_block_bytes = 0;
-  std::vector<uint32_t> dev_sizes;     // per tile: PDD bytes and Residual entries of the device image
-  size_t dir_offset = 0, blocks_offset = 0;
+  // Layout of the device image, computed on first use (tl3_device_bytes, tl3_pack, tl3_upload,
+  // tl3_stats) under `layout_mu`, so that calls that take a const handle may share it between
+  // threads; `layout_ready` is set last.
+  mutable std::mutex layout_mu;
+  mutable std::atomic<bool> layout_ready{false};
+  mutable size_t device_bytes = 0;
+  mutable uint32_t max_block_bytes = 0;
+  mutable std::vector<uint32_t> dev_sizes;   // per tile: PDD bytes and Residual entries of the device image
+  mutable size_t dir_offset = 0, blocks_offset = 0;
 
-  // last launch geometry
-  mutable int last_ctas = 0, last_stages = 0, last_smem = 0;
+  // last launch geometry (reporting only)
+  mutable std::atomic<int> last_ctas{0}, last_stages{0}, last_smem{0};
 };
 
 namespace tl3 {
@@ -69,7 +76,7 @@ struct DirEntry {
   uint32_t res_cnt;
 };
 
-size_t plan_device_layout(tl3_matrix* m);                 // fills device_bytes, offsets, max block
+size_t plan_device_layout(const tl3_matrix* m);           // fills device_bytes, offsets, max block (once, thread-safe)
 void pack_device_blob(const tl3_matrix* m, uint8_t* out); // out: device_bytes bytes, host
 
 void set_cuda_error(int e);

@@ -237,9 +237,11 @@ void for_each_tile(const tl3_matrix* m, F&& f) {
 
 }  // namespace
 
-size_t plan_device_layout(tl3_matrix* m) {
+size_t plan_device_layout(const tl3_matrix* m) {
   if (m->p.tile_m != kTileM || m->p.tile_k != kTileK) return 0;   // the device image exists for 128 x 128 tiles only
-  if (m->device_bytes) return m->device_bytes;
+  if (m->layout_ready.load(std::memory_order_acquire)) return m->device_bytes;
+  std::lock_guard<std::mutex> lock(m->layout_mu);
+  if (m->layout_ready.load(std::memory_order_relaxed)) return m->device_bytes;
   m->dev_sizes.assign(static_cast<size_t>(m->n_tiles) * 2, 0);
   for_each_tile(m, [&](int64_t t, const TileCode& tc) {
     m->dev_sizes[2 * t] = tc.pdd_len;
@@ -258,6 +260,7 @@ size_t plan_device_layout(tl3_matrix* m) {
   }
   m->max_block_bytes = max_block;
   m->device_bytes = (off + 255) / 256 * 256;
+  m->layout_ready.store(true, std::memory_order_release);
   return m->device_bytes;
 }
 

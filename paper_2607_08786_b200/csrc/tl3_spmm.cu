@@ -25,6 +25,7 @@
 #include <cuda_runtime.h>
 #include <cuda_fp16.h>
 
+#include <atomic>
 #include <cstdint>
 #include <cstring>
 #include <mutex>
@@ -67,7 +68,7 @@ constexpr uint32_t kColMetaT = 128;       // + 4 * (W_r buffer): metadata of W_t
 constexpr uint32_t kColMetaR = 152;       // two columns of 0xEEEEEEEE
 constexpr uint32_t kSmemLimit = 232448;   // 227 KB
 constexpr uint32_t kBarrierBytes = 1024;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per kernel
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s without progress, per wait
 #ifndef TL3_TRYWAIT_HINT_NS
 #define TL3_TRYWAIT_HINT_NS 20000u
 #endif
@@ -76,7 +77,7 @@ constexpr uint32_t kTryWaitHintNs = TL3_TRYWAIT_HINT_NS;     // how long one bar
 // status codes written to the workspace status word (0 = ok)
 enum : uint32_t {
   kStProducer = 1, kStDecodeFull = 2, kStDecodeWrFree = 3, kStMmaDecoded = 4, kStMmaAccEmpty = 5,
-  kStEpilogueAccFull = 6, kStDrain = 7, kStClearWrFree = 8, kStDecodeWrReady = 9, kStEpilogueTail = 10, kStEpilogueFlags = 11,
+  kStEpilogueAccFull = 6, kStDrain = 7, kStClearWrFree = 8, kStDecodeWrReady = 9, kStEpilogueTail = 10, kStEpilogueFlags = 11, kStMmaX = 12,
   kStBadBlock = 16           // a block's lengths or a decoded position were out of range (+ detail in bits 8..)
 };
 
@@ -97,22 +98,29 @@ struct KernelArgs {
   uint32_t x_offset;         // offset of the X tile inside a stage, multiple of 1024
   int num_stages;
   int num_wr;                // W_r buffers (4 or 5)
-  long long* timing;         // phase-timing buffer (debug builds), else null
+  uint32_t opts;             // kOpt* bits
+  long long* timing;         // time-stamp records (debug builds), else null
 };
 
-// Optional per-role phase timing (build with -DTL3_PHASE_TIMING): CTA 0 adds the clock cycles it
-// spends between TL3_TACC marks into a buffer set with tl3_debug_set_timing_buffer().
-#ifdef TL3_PHASE_TIMING
+// Launch options (chosen by the launcher, see tl3_tuning):
+//   kOptSplitX  the X tile of a stage completes on a barrier of its own, so that the decode of a
+//               block starts when the block is there, whether or not the kernel before this one
+//               (which may still be producing X) has finished; the MMA warp waits for both
+enum : uint32_t { kOptSplitX = 1u };
+
+// Optional per-CTA time stamps (build with -DTL3_CTA_STAMPS): one thread of a role writes the
+// SM's cycle counter into record `blockIdx.x` of the buffer set with tl3_debug_set_timing_buffer()
+// (plus the global timer once, at entry, read by a warp that idles then -- the read takes
+// microseconds -- to line the CTAs of different SMs up).  Compiled out of the product.
+#ifdef TL3_CTA_STAMPS
 static long long* g_timing_buffer = nullptr;
-#define TL3_T0() long long tacc_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long tprev_ = clock64();
-#define TL3_TACC(k) { const long long tn_ = clock64(); tacc_[k] += tn_ - tprev_; tprev_ = tn_; }
-#define TL3_TDUMP(base) { if (a.timing && blockIdx.x == 0) for (int q_ = 0; q_ < 8; ++q_) a.timing[(base) + q_] = tacc_[q_]; }
-#define TL3_STAMP(tile, k) { if (a.timing && blockIdx.x == 0 && (tile) >= 18 && (tile) < 26) a.timing[200 + 8 * ((tile) - 18) + (k)] = clock64(); }
+static int g_timing_launch = 0;
+__device__ __forceinline__ long long clock_now() { long long c; asm volatile("mov.u64 %0, %%clock64;" : "=l"(c) :: "memory"); return c; }
+#define TL3_GT(k) { if (a.timing) a.timing[blockIdx.x * 16 + (k)] = clock_now(); }
+#define TL3_GV(k, v) { if (a.timing) a.timing[blockIdx.x * 16 + (k)] = static_cast<long long>(v); }
 #else
-#define TL3_STAMP(tile, k) {}
-#define TL3_T0() {}
-#define TL3_TACC(k) {}
-#define TL3_TDUMP(base) {}
+#define TL3_GT(k) {}
+#define TL3_GV(k, v) {}
 #endif
 
 // ---------------------------------------------------------------------------------------------
@@ -151,21 +159,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return done != 0;
 }
 
-// Shared state every wait looks at: the abort flag (set by whoever gives up first), the status
-// word in global memory and the kernel's start time.
+// Shared state every wait looks at: the abort flag (set by whoever gives up first) and the
+// status word in global memory.
 struct WaitCtx {
   volatile int* abort_flag;
   unsigned int* status;
-  unsigned long long t0;
 };
 
 // Bounded wait.  Returns false if the CTA is aborting (this or another waiter ran out of time).
+// The limit runs from the moment THIS wait began to look slow (its sixteenth unsuccessful probe), not
+// from the start of the kernel: a wait that completes is progress, so a long launch, or one whose
+// context was switched out for a while earlier on, does not use up the allowance of later waits.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w, uint32_t code) {
+  unsigned long long t_slow = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 15u) == 15u) {
       if (*w.abort_flag) return false;
-      if (global_timer() - w.t0 > kWaitLimitNs) {
+      const unsigned long long now = global_timer();
+      if (t_slow == 0) t_slow = now;
+      if (now - t_slow > kWaitLimitNs) {
         atomicCAS(w.status, 0u, code);
         *w.abort_flag = 1;
         return false;
@@ -373,15 +386,19 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   const int NW = a.num_wr;
   uint8_t* wr_base = smem + static_cast<size_t>(S) * a.stage_stride;           // NW x 16 KB
   uint8_t* bar_base = wr_base + NW * kWrBytes;
-  // barrier block: full[8] mma_done[8] decoded[8] acc_full[2] acc_empty[2] | tmem slot | flags | wr_ready[5] wr_free[5]
+  // barrier block: full[8] mma_done[8] decoded[8] acc_full[2] acc_empty[2] | tmem slot | flags | tail | wr_ready[5] wr_free[5] | x_full[8]
   uint64_t* bars = reinterpret_cast<uint64_t*>(bar_base);
   const uint32_t bar_full = smem_u32(bars), bar_mma = smem_u32(bars + 8), bar_dec = smem_u32(bars + 16);
   const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26), bar_wrready = smem_u32(bars + 44), bar_wrfree = smem_u32(bars + 49);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 32);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 33);
   const uint32_t bar_tail = smem_u32(bars + 36);               // partial sums fetched into the idle stages at the very end
+  const uint32_t bar_xfull = smem_u32(bars + 56);              // [8] X tile of a stage (kOptSplitX)
+  const bool split_x = (a.opts & kOptSplitX) != 0u;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) { TL3_GT(0) }
+  if (tid == kEpilogueWarp0 * 32) { TL3_GT(1) TL3_GV(14, global_timer()) }
   const long long T = a.total_tiles, G = gridDim.x;
   const long long t_begin = range_begin(blockIdx.x, T, G), t_end = range_begin(blockIdx.x + 1, T, G);
   const int n_tiles = static_cast<int>(t_end - t_begin);
@@ -397,6 +414,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_mma + 8 * s, 1);
       mbar_init(bar_dec + 8 * s, 128);
+      mbar_init(bar_xfull + 8 * s, 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar_accfull + 8 * b, 1);
@@ -422,7 +440,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const WaitCtx wctx{abort_flag, a.status, global_timer()};
+  const WaitCtx wctx{abort_flag, a.status};
   pdl_launch_dependents();
 
   if (warp == kProducerWarp) {
@@ -431,12 +449,12 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     // Directory entries are read 32 at a time (one per lane) and broadcast with shuffles.
     // The weight blocks never depend on the kernel that ran before this one, X may: the blocks of
     // the first S tiles are requested at once, then the warp waits for the predecessor, then X.
+    constexpr uint32_t kXBytes = 128u * NPAD * 2u;
     int issued = 0, s = 0, kt = kt_begin;
     uint32_t ph = 0;                                            // phase of the stage's current use
     uint32_t stage = smem_base;
     bool alive = true;
     const int pre = n_tiles < S ? n_tiles : S;                  // tiles whose stages are free at the start
-    TL3_T0()
     for (int base = 0; base < n_tiles && alive; base += 32) {
       uint4 mine = dir_first;
       if (base > 0) {
@@ -450,52 +468,54 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
           const uint8_t* src = a.blob + static_cast<size_t>(off16) * 16;
           const uint32_t st = smem_base + static_cast<uint32_t>(j) * a.stage_stride, full = bar_full + 8 * j;
           if (elect_one()) {
-            mbar_arrive_expect_tx(full, bytes + 128u * NPAD * 2u);
+            mbar_arrive_expect_tx(full, split_x ? bytes : bytes + kXBytes);
             bulk_copy_g2s(st, src, bytes, full);
           }
           __syncwarp();
         }
+        if (lane == 0) { TL3_GT(2) }
         pdl_wait();
+        if (lane == 0) { TL3_GT(3) }
       }
       for (int j = 0; j < cnt; ++j) {
         const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.x, j), bytes = __shfl_sync(0xFFFFFFFFu, mine.y, j);
         const int i = base + j;
-        TL3_TACC(0)
         if (i >= S) alive = __all_sync(0xFFFFFFFFu, mbar_wait(bar_mma + 8 * s, ph ^ 1u, wctx, kStProducer));
-        TL3_TACC(1)
         if (!alive) break;
-        if (lane == 0) TL3_STAMP(i, 0)
         const uint32_t full = bar_full + 8 * s;
+        const uint32_t xbar = split_x ? bar_xfull + 8 * s : full;
         const uint8_t* src = a.blob + static_cast<size_t>(off16) * 16;
         if (elect_one()) {
           if (i >= pre) {
-            mbar_arrive_expect_tx(full, bytes + 128u * NPAD * 2u);
+            mbar_arrive_expect_tx(full, split_x ? bytes : bytes + kXBytes);
             bulk_copy_g2s(stage, src, bytes, full);
           }
+          if (split_x) mbar_arrive_expect_tx(xbar, kXBytes);
           if (XT) {
-            tma_load_2d(stage + a.x_offset, &x_map, kt * kTileK, 0, full);
-            tma_load_2d(stage + a.x_offset + NPAD * 128u, &x_map, kt * kTileK + 64, 0, full);
+            tma_load_2d(stage + a.x_offset, &x_map, kt * kTileK, 0, xbar);
+            tma_load_2d(stage + a.x_offset + NPAD * 128u, &x_map, kt * kTileK + 64, 0, xbar);
           } else {
-            tma_load_2d(stage + a.x_offset, &x_map, 0, kt * kTileK, full);
+            tma_load_2d(stage + a.x_offset, &x_map, 0, kt * kTileK, xbar);
           }
-          TL3_STAMP(i, 1)
         }
         __syncwarp();
+        if (lane == 0) { if (i == 0) { TL3_GT(4) } if (i == n_tiles - 1) { TL3_GT(8) } }
         issued = i + 1;
         stage += a.stage_stride;
         if (++s == S) { s = 0; ph ^= 1u; stage = smem_base; }
         if (++kt == a.tiles_k) kt = 0;
       }
     }
-    if (lane == 0) TL3_TDUMP(0)
     if (lane == 0 && *abort_flag) {
       // let the copies still in flight land before the CTA goes away
       const int first = issued > S ? issued - S : 0;
       for (int i = first; i < issued; ++i) {
-        const uint32_t full = bar_full + 8 * (i % S);
         const unsigned long long t1 = global_timer();
-        while (!mbar_try_wait(full, (i / S) & 1)) {
-          if (global_timer() - t1 > kWaitLimitNs / 4) { atomicCAS(a.status, 0u, (uint32_t)kStDrain); break; }
+        for (int which = 0; which < (split_x ? 2 : 1); ++which) {
+          const uint32_t bar = (which ? bar_xfull : bar_full) + 8 * (i % S);
+          while (!mbar_try_wait(bar, (i / S) & 1)) {
+            if (global_timer() - t1 > kWaitLimitNs / 4) { atomicCAS(a.status, 0u, (uint32_t)kStDrain); break; }
+          }
         }
       }
     }
@@ -544,18 +564,15 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     const uint32_t w_lo0 = (smem_u32(wr_base) >> 4) | kLboOne;
     int seg = 0, s = 0, kt = kt_begin, wb = 0;
     uint32_t ph = 0, a_lo = a_lo0;
-    TL3_T0()
     for (int i = 0; i < n_tiles; ++i) {
       const bool first_of_seg = (i == 0) || (kt == 0);
       const bool last_of_seg = (i == n_tiles - 1) || (kt == a.tiles_k - 1);
       const int b = seg & 1;
       bool ok = true;
       if (first_of_seg && (seg >> 1) >= 1) ok = mbar_wait(bar_accempty + 8 * b, ((seg >> 1) - 1) & 1, wctx, kStMmaAccEmpty);
-      TL3_TACC(0)
       ok = ok && mbar_wait(bar_dec + 8 * s, ph, wctx, kStMmaDecoded);
-      TL3_TACC(1)
+      if (split_x) ok = ok && mbar_wait(bar_xfull + 8 * s, ph, wctx, kStMmaX);
       if (!__all_sync(0xFFFFFFFFu, ok)) break;
-      if (lane == 0) TL3_STAMP(i, 4)
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(b * NPAD);
       const uint32_t e_t = tmem_base + kColMetaT + 4 * wb, e_r = tmem_base + kColMetaR;
@@ -574,15 +591,13 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         if (last_of_seg) umma_commit(acc_bar);
       }
       __syncwarp();
-      if (lane == 0) TL3_STAMP(i, 5)
-      TL3_TACC(2)
+      if (lane == 0) { if (i == 0) { TL3_GT(7) } if (i == n_tiles - 1) { TL3_GT(9) } }
       if (last_of_seg) ++seg;
       a_lo += stride16;
       if (++s == S) { s = 0; ph ^= 1u; a_lo = a_lo0; }
       if (++kt == a.tiles_k) kt = 0;
       if (++wb == NW) wb = 0;
     }
-    if (lane == 0) TL3_TDUMP(8)
   } else if (warp >= kDecodeWarp0 && warp < kEpilogueWarp0) {
     // ------------------------------------------------------------------ decode (Algorithm 1)
     const int g = (warp - kDecodeWarp0) >> 2;
@@ -596,9 +611,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     int wb = g % NW, use = g / NW;                              // W_r buffer of tile i and how often it was filled before
     int s = g;                                                  // g < AG <= S
     uint32_t ph = 0;
-    TL3_T0()
     for (int i = g, j = 0; g < AG && i < n_tiles; i += AG, ++j) {
-      TL3_TACC(0)
       // Warps of a group do not wait for each other.  The packed block lists chains longest
       // first, so the four warps get blocks of different length; the block a warp takes rotates
       // from tile to tile to even the load out.
@@ -610,9 +623,8 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       // wait on the stage's `full` barrier unambiguous (loads may complete out of order, and a
       // parity wait cannot tell "two phases back" from "done").
       bool ok = mbar_wait(bar_wrready + 8 * wb, use & 1, wctx, kStDecodeWrReady);
-      TL3_TACC(1)
       ok = ok && mbar_wait(bar_full + 8 * s, ph, wctx, kStDecodeFull);
-      TL3_TACC(2)
+      if (r == 0 && i == 0) { TL3_GT(5) }
       const uint32_t stage = smem_base + static_cast<uint32_t>(s) * a.stage_stride;
       uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0, span = 0, hdr = 0xFFFFFFFFu, pdd_len = 0, res_cnt = 0;
       if (ok) {
@@ -623,14 +635,12 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         res_cnt = lds_u32(stage + kInfoOff + 4);
       }
       if (!__all_sync(0xFFFFFFFFu, ok)) break;
-      if (r == 0) TL3_STAMP(i, 2)
       // metadata -> tensor memory (4 columns of this group)
       {
         asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
                      ::"r"(tmem_base + lane_base + kColMetaT + 4 * wb), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
       }
       const uint32_t n_words = span;
-      TL3_TACC(4)
       uint32_t bad = 0;
       const uint32_t room = a.x_offset - kPddOff;               // bytes a block may use after its fixed part
       const bool lens_ok = pdd_len <= room && res_cnt <= room / 4 && ((pdd_len + 3u) & ~3u) + 4u * res_cnt <= room &&
@@ -638,7 +648,6 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       if (lens_ok) decode_chain(stage, wr, hdr, stage + kPddOff + cr * 4, n_words, &bad);
       else bad = 3u;
       __syncwarp();
-      TL3_TACC(5)
       // Residual layer: (position, value) entries go to W_r too
       if (lens_ok) {
         const uint32_t res = stage + kPddOff + ((pdd_len + 3u) & ~3u);
@@ -649,19 +658,17 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         }
       }
       if (bad) atomicCAS(a.status, 0u, kStBadBlock | (bad << 8) | (static_cast<uint32_t>(i) << 12));
-      TL3_TACC(6)
       fence_proxy_async_smem();                                   // generic-proxy writes -> MMA reads
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       tc_fence_before();
       mbar_arrive(bar_dec + 8 * s);
-      if (r == 0) TL3_STAMP(i, 3)
-      TL3_TACC(7)
+      if (r == 0 && i == 0) { TL3_GT(6) }
+      if (r == 0 && i == n_tiles - 1) { TL3_GT(15) }
       s += AG;
       while (s >= S) { s -= S; ph ^= 1u; }
       wb += AG;
       while (wb >= NW) { wb -= NW; ++use; }
     }
-    if (lane == 0) TL3_TDUMP(16 + 8 * (warp - kDecodeWarp0))
   } else if (warp >= kEpilogueWarp0) {
     // ------------------------------------------------------------------ epilogue
     const int et = tid - kEpilogueWarp0 * 32;                    // 0..127 = row of the tile = tensor-memory lane
@@ -669,9 +676,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     int seg = 0;
     long long t = t_begin;
     pdl_wait();   // Y, the partial sums and their flags may still be in use by the previous kernel
-    TL3_T0()
     while (t < t_end) {
-      TL3_TACC(0)
       const int mt = static_cast<int>(t / a.tiles_k);
       const long long row_tile_begin = static_cast<long long>(mt) * a.tiles_k, row_tile_end = row_tile_begin + a.tiles_k;
       const long long seg_end = row_tile_end < t_end ? row_tile_end : t_end;
@@ -687,7 +692,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       const bool reducer = !complete && static_cast<int>(blockIdx.x) == c_first;
       const int n_others = c_last - c_first;
       if (!named_bar_all(1 + kGroups, 128, mbar_wait(bar_accfull + 8 * b, (seg >> 1) & 1, wctx, kStEpilogueAccFull))) break;
-      TL3_TACC(1)
+      if (et == 0 && seg_end == t_end) { TL3_GT(10) TL3_GV(13, reducer ? n_others : (complete ? 0 : -1)) }
       tc_fence_after();
       constexpr int CH = NPAD < 32 ? NPAD : 32;                 // columns handled per round (register budget)
       __half* y = XT ? a.Y + row : a.Y + static_cast<long long>(row) * a.ldy;   // XT: element (row, c) at y[c * ldy]
@@ -749,6 +754,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
               const int c_id = c_first + 1 + k;
               sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
             }
+            unsigned long long t_slow = 0;                        // limit counted from when this poll began to look slow
             for (uint32_t it = 0; __any_sync(0xFFFFFFFFu, pending); ++it) {
               if (pending) {
                 unsigned int up;
@@ -764,7 +770,9 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
                 }
               }
               if ((it & 15u) == 15u) {
-                const bool out = *abort_flag != 0 || global_timer() - wctx.t0 > kWaitLimitNs;
+                const unsigned long long now = global_timer();
+                if (t_slow == 0) t_slow = now;
+                const bool out = *abort_flag != 0 || now - t_slow > kWaitLimitNs;
                 if (__any_sync(0xFFFFFFFFu, out)) {
                   if (et == 0) { atomicCAS(a.status, 0u, static_cast<uint32_t>(kStEpilogueFlags)); *abort_flag = 1; }
                   ok = false;
@@ -810,7 +818,6 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         }
         tc_fence_before();
         mbar_arrive(bar_accempty + 8 * b);
-        TL3_TACC(2)
         ++seg;
         t = seg_end;
         continue;
@@ -834,16 +841,16 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         named_bar_sync(1 + kGroups, 128);
         if (et == 0) asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(a.flags + slot), "r"(1u) : "memory");
       }
-      TL3_TACC(2)
       ++seg;
       t = seg_end;
     }
-    if (et == 0) TL3_TDUMP(160)
   }
 
   // ------------------------------------------------------------------ teardown
+  if (tid == kEpilogueWarp0 * 32) { TL3_GT(11) }
   tc_fence_before();
   __syncthreads();
+  if (tid == kEpilogueWarp0 * 32) { TL3_GT(12) }
   if (warp == kAllocWarp) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
@@ -862,7 +869,7 @@ __global__ void bounded_wait_probe_kernel(unsigned int* status, unsigned int* ou
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  const WaitCtx w{&abort_flag, status, global_timer()};
+  const WaitCtx w{&abort_flag, status};
   const bool completed = mbar_wait(smem_u32(&bar), 0, w, kStProducer);
   if (threadIdx.x == 0) *outcome = completed ? 1u : 2u;
 }
@@ -923,12 +930,24 @@ static WorkspaceLayout workspace_layout(const tl3_matrix* m, int n_pad, int sm_c
   return w;
 }
 
+// Process-wide launch tuning (tl3_set_tuning); the default is what measured best on B200.
+static std::atomic<int> g_decode_before_x{TL3_DEFAULT_DECODE_BEFORE_X};
+
 template <int NPAD, bool XT>
 static int launch(const CUtensorMap& map, const KernelArgs& args, int grid, uint32_t smem_bytes, cudaStream_t stream) {
-  static bool configured = false;   // per template instance; same value every time
-  if (!configured) {
-    TL3_CUDA(cudaFuncSetAttribute(tl3_spmm_kernel<NPAD, XT>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemLimit)));
-    configured = true;
+  // The opt-in to more than 48 KB of dynamic shared memory is a property of the function on ONE
+  // device: it is set once per device and template instance.
+  {
+    int dev = 0;
+    TL3_CUDA(cudaGetDevice(&dev));
+    static std::mutex mu;
+    static std::vector<char> configured;
+    std::lock_guard<std::mutex> lock(mu);
+    if (static_cast<size_t>(dev) >= configured.size()) configured.resize(dev + 1, 0);
+    if (!configured[dev]) {
+      TL3_CUDA(cudaFuncSetAttribute(tl3_spmm_kernel<NPAD, XT>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemLimit)));
+      configured[dev] = 1;
+    }
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
@@ -951,13 +970,13 @@ extern "C" {
 
 size_t tl3_device_bytes(const tl3_matrix* m) {
   if (!m) return 0;
-  return tl3::plan_device_layout(const_cast<tl3_matrix*>(m));
+  return tl3::plan_device_layout(m);
 }
 
 int tl3_pack(const tl3_matrix* m, void* host_buf, size_t bytes) {
   if (!m || !host_buf) return TL3_ERR_INVALID_ARG;
   if (m->p.tile_m != tl3::kTileM || m->p.tile_k != tl3::kTileK) return TL3_ERR_UNSUPPORTED;
-  if (bytes < tl3::plan_device_layout(const_cast<tl3_matrix*>(m))) return TL3_ERR_INVALID_ARG;
+  if (bytes < tl3::plan_device_layout(m)) return TL3_ERR_INVALID_ARG;
   tl3::pack_device_blob(m, static_cast<uint8_t*>(host_buf));
   return TL3_OK;
 }
@@ -1067,8 +1086,13 @@ static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, 
   args.x_offset = block_area;
   args.num_stages = stages;
   args.num_wr = num_wr;
-#ifdef TL3_PHASE_TIMING
-  args.timing = g_timing_buffer;
+  // Decoding ahead of X pays where a launch is short (a tile or a few per CTA: most of its time is
+  // the start) and measured level or slightly worse on longer ones.
+  const int dbx = g_decode_before_x.load(std::memory_order_relaxed);
+  const long long tiles_per_cta = (total + grid - 1) / grid;
+  args.opts = (dbx < 0 || tiles_per_cta <= dbx) ? kOptSplitX : 0u;
+#ifdef TL3_CTA_STAMPS
+  args.timing = g_timing_buffer ? g_timing_buffer + static_cast<long long>(g_timing_launch++ % 64) * 148 * 16 : nullptr;
 #else
   args.timing = nullptr;
 #endif
@@ -1226,6 +1250,22 @@ int tl3_last_launch(const tl3_matrix* m, int* ctas, int* stages, int* smem_bytes
 
 int tl3_last_cuda_error(void) { return tl3::g_last_cuda_error; }
 
+int tl3_get_tuning(tl3_tuning* out) {
+  if (!out) return TL3_ERR_INVALID_ARG;
+  out->decode_before_x = tl3::g_decode_before_x.load();
+  return TL3_OK;
+}
+
+int tl3_set_tuning(const tl3_tuning* t) {
+  if (!t) {
+    tl3::g_decode_before_x = TL3_DEFAULT_DECODE_BEFORE_X;
+    return TL3_OK;
+  }
+  if (t->decode_before_x < -1) return TL3_ERR_INVALID_ARG;
+  tl3::g_decode_before_x = t->decode_before_x;
+  return TL3_OK;
+}
+
 int tl3_selftest_bounded_wait(void* workspace, void* stream) {
   if (!workspace) return TL3_ERR_INVALID_ARG;
   unsigned int* words = static_cast<unsigned int*>(workspace);
@@ -1234,8 +1274,8 @@ int tl3_selftest_bounded_wait(void* workspace, void* stream) {
   return TL3_OK;
 }
 
-#ifdef TL3_PHASE_TIMING
-void tl3_debug_set_timing_buffer(long long* device_ptr) { tl3::g_timing_buffer = device_ptr; }
+#ifdef TL3_CTA_STAMPS
+void tl3_debug_set_timing_buffer(long long* device_ptr) { tl3::g_timing_buffer = device_ptr; tl3::g_timing_launch = 0; }   // 64 x 148 x 16 int64
 #endif
 
 }  // extern "C"

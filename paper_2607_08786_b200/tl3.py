@@ -28,7 +28,7 @@ _CANONICAL_DTYPES = (np.uint16, np.uint8, np.uint16, np.uint16, np.uint8, np.uin
 SYMBOLS = ("tl3_encode", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_deserialize",
            "tl3_free", "tl3_device_bytes", "tl3_pack", "tl3_upload", "tl3_workspace_bytes", "tl3_workspace_init",
            "tl3_spmm", "tl3_spmm_ex", "tl3_spmm_nt", "tl3_spmm_host", "tl3_spmm_host_async", "tl3_spmm_static_scratch", "tl3_static_scratch_status", "tl3_status", "tl3_status_word", "tl3_selftest_bounded_wait", "tl3_last_launch", "tl3_strerror",
-           "tl3_last_cuda_error")
+           "tl3_last_cuda_error", "tl3_get_tuning", "tl3_set_tuning")
 
 
 class Tl3Error(RuntimeError):
@@ -42,6 +42,10 @@ class Tl3Error(RuntimeError):
 
 class Params(ctypes.Structure):
     _fields_ = [("tile_m", ctypes.c_int32), ("tile_k", ctypes.c_int32), ("maxd", ctypes.c_int32)]
+
+
+class Tuning(ctypes.Structure):
+    _fields_ = [("decode_before_x", ctypes.c_int32)]
 
 
 class Epilogue(ctypes.Structure):
@@ -101,6 +105,8 @@ def lib() -> ctypes.CDLL:
         L.tl3_strerror.argtypes = [ci]
         L.tl3_strerror.restype = ctypes.c_char_p
         L.tl3_last_cuda_error.argtypes = []
+        L.tl3_get_tuning.argtypes = [ctypes.POINTER(Tuning)]
+        L.tl3_set_tuning.argtypes = [ctypes.POINTER(Tuning)]
         for name in SYMBOLS:
             fn = getattr(L, name)
             if name not in ("tl3_free", "tl3_device_bytes", "tl3_workspace_bytes", "tl3_strerror"):
@@ -337,3 +343,21 @@ class Matrix:
 
 def encode(W, **kw) -> Matrix:
     return Matrix.encode(W, **kw)
+
+
+def get_tuning() -> dict:
+    """The process-wide launch tuning (``tl3_get_tuning``)."""
+    t = Tuning()
+    _check(lib().tl3_get_tuning(ctypes.byref(t)), "tl3_get_tuning")
+    return {n: int(getattr(t, n)) for n, _ in Tuning._fields_}
+
+
+def set_tuning(**kw) -> None:
+    """``set_tuning()`` restores the defaults; keywords override single fields of the current tuning."""
+    if not kw:
+        _check(lib().tl3_set_tuning(None), "tl3_set_tuning")
+        return
+    cur = get_tuning()
+    cur.update(kw)
+    t = Tuning(**cur)
+    _check(lib().tl3_set_tuning(ctypes.byref(t)), "tl3_set_tuning")

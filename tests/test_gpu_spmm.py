@@ -200,7 +200,7 @@ def test_workspace_is_left_cleared_and_can_serve_another_matrix(tl3, oracle_mod)
         check(oracle_mod, W, X, Y.cpu().numpy(), with_oracle_spmm=False)
 
 
-def test_thousands_of_back_to_back_launches(tl3):
+def test_thousands_of_back_to_back_launches(tl3, oracle_mod):
     """Five different launches in one CUDA graph, replayed without host synchronisation: every
     replay must leave the status words clear and reproduce the first result bit for bit (the
     pipeline's barrier protocol must not depend on how loads happen to be ordered in time)."""
@@ -210,13 +210,15 @@ def test_thousands_of_back_to_back_launches(tl3):
              wl.Case(0, "e", 3000, 3000, 24, 5, 0.7, "magnitude")]
     L = []
     for c in cases:
-        m = tl3.encode(c.make_W())
+        W, X = c.make_W(), c.make_X()
+        m = tl3.encode(W)
         m.upload()
-        Xd = device_X(c.make_X())
+        Xd = device_X(X)
         ws = m.new_workspace(c.N)
         Y = torch.empty((c.M, c.N), dtype=torch.float16, device="cuda")
         m.spmm(Xd, Y, workspace=ws)
         torch.cuda.synchronize()
+        check(oracle_mod, W, X, Y.cpu().numpy())             # the result every replay is compared with
         L.append((c, m, Xd, Y, ws, Y.clone()))
 
     def step():
@@ -235,7 +237,7 @@ def test_thousands_of_back_to_back_launches(tl3):
             assert torch.equal(Y, ref), c.name
 
 
-def test_concurrent_launches_on_several_streams(tl3):
+def test_concurrent_launches_on_several_streams(tl3, oracle_mod):
     """The same five launches forked over three streams inside one CUDA graph, so that kernels of
     different streams share the GPU (a kernel moves in as another moves out, and CTAs of a launch
     may still be waiting for an SM while its reducers already collect): results and status as in
@@ -246,13 +248,15 @@ def test_concurrent_launches_on_several_streams(tl3):
              wl.Case(0, "e", 3000, 3000, 24, 5, 0.7, "magnitude")]
     L = []
     for c in cases:
-        m = tl3.encode(c.make_W())
+        W, X = c.make_W(), c.make_X()
+        m = tl3.encode(W)
         m.upload()
-        Xd = device_X(c.make_X())
+        Xd = device_X(X)
         ws = m.new_workspace(c.N)
         Y = torch.empty((c.M, c.N), dtype=torch.float16, device="cuda")
         m.spmm(Xd, Y, workspace=ws)
         torch.cuda.synchronize()
+        check(oracle_mod, W, X, Y.cpu().numpy())             # the result every replay is compared with
         L.append((c, m, Xd, Y, ws, Y.clone()))
     side = [torch.cuda.Stream() for _ in range(2)]
 
@@ -533,3 +537,63 @@ def test_full_size_configs_sampled(tl3, oracle_mod, config):
         m.close()
         del Xd, Y, ws
         torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("N", [16, 32])
+def test_long_tile_ranges_are_exact_on_small_integers(tl3, oracle_mod, N):
+    """20480 x 5120 in the benchmark's launch configuration: 43 tiles per CTA, so the producer reads
+    its directory in two batches and every stage, W_r buffer and accumulator barrier wraps many
+    times.  With small integers every partial sum is exact in fp32 whatever the order, so ALL rows
+    must equal the oracle's format walk and the exact product bit for bit: one dropped or doubled
+    weight anywhere shows."""
+    rng = np.random.default_rng(2024 + N)
+    M, K = 20480, 5120
+    W = np.where(rng.random((M, K)) < 0.5, rng.integers(-4, 5, (M, K)), 0).astype(np.float16)
+    X = rng.integers(-3, 4, (K, N)).astype(np.float16)
+    Y, m = run_gpu(tl3, W, X)
+    assert m.last_launch()["ctas"] == 148
+    exact = W.astype(np.float64) @ X.astype(np.float64)            # integers below 2^53: exact
+    assert np.array_equal(Y.view(np.uint16), exact.astype(np.float16).view(np.uint16))
+    assert np.array_equal(Y.view(np.uint16), oracle_mod.spmm(oracle_mod.encode(W), X))
+
+
+@pytest.mark.parametrize("config,index", [(2, 5), (3, 4), (4, 2), (5, 3)])
+def test_full_size_all_rows(tl3, oracle_mod, config, index):
+    """One shape of every benchmark configuration, EVERY row against the float64 definition (in row
+    blocks to bound memory) and against the oracle's format walk, whose tolerance is tight enough
+    to see a single dropped weight."""
+    import torch
+    case = list(wl.config_cases(config))[index]
+    W, X = case.make_W(), case.make_X()
+    m = tl3.encode(W)
+    m.upload()
+    ws = m.new_workspace(case.N)
+    Y = m.spmm(torch.from_numpy(X).cuda(), workspace=ws)
+    torch.cuda.synchronize()
+    assert m.status(ws) == tl3.OK
+    Yh = Y.cpu().numpy()
+    Yo = oracle_mod.spmm(oracle_mod.encode(W), X).view(np.float16).astype(np.float64)
+    for r0 in range(0, case.M, 2048):
+        r1 = min(case.M, r0 + 2048)
+        Yref, bound = oracle_mod.dense_fp64(W[r0:r1], X)
+        y = Yh[r0:r1].astype(np.float64)
+        assert np.all(np.abs(y - Yref) <= oracle_mod.tolerance(bound)), (case.name, r0)
+        assert np.all(np.abs(y - Yo[r0:r1]) <= 2.0**-9 * np.abs(Yo[r0:r1]) + 1e-4 * bound + 1e-6), (case.name, r0)
+
+
+def test_decoding_ahead_of_x_changes_no_bit(tl3):
+    """The launch option that lets the decode warps start on a block before its X tile has arrived
+    only moves a wait: results are bit-identical with it forced on and off."""
+    import torch
+    outs = []
+    case = wl.Case(0, "dbx", 2560, 3072, 24, 9, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    try:
+        for setting in (0, -1):
+            tl3.set_tuning(decode_before_x=setting)
+            Y, _ = run_gpu(tl3, W, X, repeats=2)
+            outs.append(Y)
+    finally:
+        tl3.set_tuning()
+    assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
+    assert tl3.get_tuning()["decode_before_x"] == 4

@@ -162,6 +162,50 @@ def test_error_codes(tl3):
     assert L.tl3_strerror(-99) == b"unknown error"
 
 
+def test_launch_tuning_round_trip(tl3):
+    L = tl3.lib()
+    assert tl3.get_tuning() == {"decode_before_x": 4}
+    try:
+        tl3.set_tuning(decode_before_x=-1)
+        assert tl3.get_tuning()["decode_before_x"] == -1
+        bad = tl3.Tuning(-2)
+        assert L.tl3_set_tuning(ctypes.byref(bad)) == tl3.ERR_INVALID_ARG
+        assert tl3.get_tuning()["decode_before_x"] == -1          # a refused setting changes nothing
+        assert L.tl3_get_tuning(None) == tl3.ERR_INVALID_ARG
+    finally:
+        tl3.set_tuning()
+    assert tl3.get_tuning() == {"decode_before_x": 4}
+
+
+def test_const_calls_on_one_handle_from_several_threads(tl3):
+    """tl3_device_bytes / tl3_stats / tl3_pack take a const handle and compute the layout of the
+    device image on first use: four threads that make that first use together must all see the same,
+    complete layout (the blob of each equals the blob packed afterwards by one thread)."""
+    import threading
+    case = wl.Case(0, "thr", 1024, 1536, 8, 31, 0.5, "magnitude")
+    m = tl3.encode(case.make_W())
+    out, errs = [None] * 4, []
+
+    def work(i):
+        try:
+            n = m.device_bytes()
+            st = m.stats()
+            assert st["device_bytes"] == n
+            out[i] = m.pack()
+        except Exception as e:                                   # pragma: no cover
+            errs.append(e)
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(4)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errs
+    ref = m.pack()
+    for o in out:
+        assert o is not None and np.array_equal(o, ref)
+
+
 def _image_offset(u):
     """Byte offset of bank-major slot u = bank << 8 | slot-in-window << 7 | row in the value image."""
     return ((u & 127) << 7) | ((u >> 6) & 0x7E)

@@ -47,6 +47,15 @@ def test_static_scratch_entry_point_matches_the_regular_one(oracle_mod):
         assert np.all(np.abs(got.astype(np.float64) - Yref64) <= tol), f"call {call}"
         # same kernel, same fixed summation order: the bits agree as well
         assert np.array_equal(got.view(np.uint16), ref.view(np.uint16)), f"call {call}"
+    # and it really obtains no device memory: after the warm-up calls above, one more call with Y
+    # already allocated leaves the device's free memory and torch's own books where they were
+    Y = torch.empty((case.M, case.N), dtype=torch.float16, device="cuda")
+    torch.cuda.synchronize()
+    free_before, booked_before = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+    rc = L.tl3_spmm_static_scratch(m._h, Xd.data_ptr(), Xd.stride(0), Y.data_ptr(), Y.stride(0), case.N, stream)
+    assert rc == tl3.OK
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before and torch.cuda.memory_allocated() == booked_before
 
 
 def test_static_scratch_refuses_what_does_not_fit():
