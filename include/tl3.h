@@ -118,6 +118,14 @@ int tl3_pack(const tl3_matrix* m, void* host_buf, size_t bytes);
  * Errors: UNSUPPORTED (tile shape other than 128 x 128), INVALID_ARG, CUDA. */
 int tl3_upload(tl3_matrix* m, void* dptr, void* stream);
 
+/* Bind a device buffer that already holds the packed blob -- the bytes of tl3_pack() copied to the
+ * device by the caller, or a device-side copy of a blob that tl3_upload() wrote -- to the handle:
+ * later tl3_spmm* calls read the weights from there.  dptr: device, >= tl3_device_bytes(),
+ * 256-byte aligned.  Nothing is copied or checked.  A launch reads the binding when it is enqueued
+ * (or captured into a CUDA graph), so one handle may serve several device copies in turn.
+ * Errors: INVALID_ARG, UNSUPPORTED (tile shape other than 128 x 128). */
+int tl3_bind(tl3_matrix* m, void* dptr);
+
 /* Scratch the kernel needs for N columns: split-K partial sums, one arrival flag per partial-sum
  * slot, a status word.  Depends on the current device's SM count.  The caller allocates it (device,
  * 256-byte aligned), clears it once with tl3_workspace_init(), and may then reuse it for any number

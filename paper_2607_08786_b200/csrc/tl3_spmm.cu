@@ -998,6 +998,14 @@ int tl3_upload(tl3_matrix* m, void* dptr, void* stream) {
   return TL3_OK;
 }
 
+int tl3_bind(tl3_matrix* m, void* dptr) {
+  if (!m || !dptr || (reinterpret_cast<uintptr_t>(dptr) & 255) != 0) return TL3_ERR_INVALID_ARG;
+  if (m->p.tile_m != tl3::kTileM || m->p.tile_k != tl3::kTileK) return TL3_ERR_UNSUPPORTED;
+  tl3::plan_device_layout(m);
+  m->dptr = dptr;
+  return TL3_OK;
+}
+
 size_t tl3_workspace_bytes(const tl3_matrix* m, int N) {
   if (!m || N < 1 || N > TL3_MAX_N) return 0;
   tl3::DeviceInfo di;

@@ -597,3 +597,27 @@ def test_decoding_ahead_of_x_changes_no_bit(tl3):
         tl3.set_tuning()
     assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
     assert tl3.get_tuning()["decode_before_x"] == 4
+
+
+def test_bind_serves_device_copies_of_the_blob(tl3, oracle_mod):
+    """A blob packed on the host and copied over by the caller, and a device-side clone of an
+    uploaded blob, give the same bits as the uploaded one; a misaligned pointer is refused."""
+    import torch
+    case = wl.Case(0, "bind", 1280, 2304, 16, 17, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    m = tl3.encode(W)
+    first = m.upload()
+    Xd = device_X(X)
+    ws = m.new_workspace(case.N)
+    Y0 = m.spmm(Xd, workspace=ws).clone()
+    check(oracle_mod, W, X, Y0.cpu().numpy())
+    packed = torch.from_numpy(m.pack()).cuda()
+    clone = first.clone()
+    first.zero_()                                               # the old binding must not be read any more
+    for blob in (packed, clone):
+        m.bind(blob)
+        Y = m.spmm(Xd, workspace=ws)
+        torch.cuda.synchronize()
+        assert m.status(ws) == tl3.OK
+        assert torch.equal(Y, Y0)
+    assert tl3.lib().tl3_bind(m._h, packed.data_ptr() + 16) == tl3.ERR_INVALID_ARG
