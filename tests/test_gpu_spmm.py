@@ -621,3 +621,16 @@ def test_bind_serves_device_copies_of_the_blob(tl3, oracle_mod):
         assert m.status(ws) == tl3.OK
         assert torch.equal(Y, Y0)
     assert tl3.lib().tl3_bind(m._h, packed.data_ptr() + 16) == tl3.ERR_INVALID_ARG
+
+
+def test_row_sharded_matrix_on_one_rank(tl3, oracle_mod):
+    """The row-split wrapper with its default per-rank product (the library on the current device);
+    with one rank its slab is the whole matrix and no collective runs."""
+    import torch
+    from paper_2607_08786_b200 import dist
+    case = wl.Case(0, "rs", 900, 1024, 16, 5, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    sh = dist.RowShardedMatrix(W)
+    Y = sh.matmul(device_X(X))
+    torch.cuda.synchronize()
+    check(oracle_mod, W, X, Y.cpu().numpy())

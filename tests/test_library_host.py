@@ -389,3 +389,58 @@ print("rank", rank, "ok")
     for rank, (p, out) in enumerate(zip(procs, outs)):
         assert p.returncode == 0, out
         assert f"rank {rank} ok" in out
+
+
+def test_row_shard_ranges():
+    from paper_2607_08786_b200 import dist
+    for M, world in ((1000, 2), (128, 4), (36864, 8), (130, 3)):
+        ranges = [dist.row_shard(M, r, world) for r in range(world)]
+        assert ranges[0][0] == 0 and ranges[-1][1] == M
+        for (a, b), (c, d) in zip(ranges[:-1], ranges[1:]):
+            assert b == c and a % 128 == 0 and c % 128 == 0      # contiguous, cut between row-tiles
+        sizes = [(b - a + 127) // 128 for a, b in ranges]
+        assert max(sizes) - min(sizes) <= 1
+
+
+def test_row_split_over_two_ranks_on_cpu():
+    """world_size 2 over gloo: one W split by rows (the 2-GPU arrangement of Sec. 5.3), X replicated,
+    all-gather of Y.  The per-rank product is a CPU stand-in (the library's own encoder and decoder
+    around a float32 matmul), so this covers the partitioning, the padding of unequal slabs and the
+    collective; the kernel itself is covered by the GPU tests."""
+    import subprocess
+    import sys
+    import socket
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    code = r"""
+import os, sys
+sys.path.insert(0, %r)
+import numpy as np, torch
+from paper_2607_08786_b200 import dist, tl3, workloads as wl
+rank, local_rank, world = dist.init_process_group("gloo")
+case = wl.Case(0, "split", 1000, 512, 8, 99, 0.5, "magnitude")      # 8 row-tiles, the last one ragged
+W, X = case.make_W(), case.make_X()
+def stand_in(slab):
+    m = tl3.encode(slab)                                              # each rank encodes only its slab
+    Wd = torch.from_numpy(m.decode().view(np.float16).astype(np.float32))
+    return lambda Xt: (Wd @ Xt.float()).half()
+sh = dist.RowShardedMatrix(W, local_product=stand_in)
+assert sh.ranges == [(0, 512), (512, 1000)], sh.ranges
+Y = sh.matmul(torch.from_numpy(X))
+ref = (torch.from_numpy(W.astype(np.float32)) @ torch.from_numpy(X.astype(np.float32))).half()
+assert Y.shape == (1000, 8) and torch.allclose(Y.float(), ref.float(), atol=2e-3, rtol=2e-3)
+dist.barrier()
+print("rank", rank, "ok")
+""" % ROOT
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE="2",
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, "-c", code], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.STDOUT, text=True))
+    outs = [p.communicate(timeout=180)[0] for p in procs]
+    for rank, (p, out) in enumerate(zip(procs, outs)):
+        assert p.returncode == 0, out
+        assert f"rank {rank} ok" in out
