@@ -6,11 +6,14 @@ only the tests, the smoke check and the CPU-baseline leg of the benchmark do.
 from .oracle import (  # noqa: F401
     Container,
     build,
+    compact_nbytes,
     decode,
     dense_fp64,
     encode,
     float_to_half,
     half_to_float,
+    residual_compact,
+    residual_expand,
     spmm,
     threads,
     tolerance,

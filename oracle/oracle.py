@@ -199,3 +199,68 @@ def half_to_float(h: int) -> float:
 
 def float_to_half(f: float) -> int:
     return int(_load().oracle_float_to_half(float(f)))
+
+
+# ---- compact form of the Residual layer ---------------------------------------------------------
+# Sec. 3.2 leaves the Residual format open ("a classic format such as CSR") because at 50 % it
+# holds under 1 % of the non-zeros.  Below 50 % sparsity it does not stay small (no tile has room
+# for more than half of its weights in the value slots), and two bytes of position per entry add
+# up.  The compact form keeps, per tile, whichever is smaller: the position list, or a bitmap over
+# the tile's tile_m * H positions of W_r (bit rho % 8 of byte rho // 8) with the values in
+# ascending position order as before.
+def residual_compact(c: Container):
+    """(res_dir, res_list, res_mask) of a container's Residual layer.
+
+    res_dir  u32[tiles][2]  {mode, off}: mode 0 = position list, off = index of the tile's first
+                            position in res_list; mode 1 = bitmap, off = byte offset of the tile's
+                            bitmap in res_mask
+    res_list u16[]          positions of the list-mode tiles, tile after tile
+    res_mask u8[]           ceil(tile_m * H / 8) bytes per bitmap-mode tile
+    A tile takes the bitmap iff it is strictly smaller than the tile's two-byte positions."""
+    H = c.tile_k // 2
+    B = (c.tile_m * H + 7) // 8
+    n_tiles = c.tile_dir.shape[0]
+    res_dir = np.zeros((n_tiles, 2), dtype=np.uint32)
+    lists, masks = [], []
+    n_list = n_mask = 0
+    for t in range(n_tiles):
+        off, cnt = int(c.tile_dir[t, 2]), int(c.tile_dir[t, 3])
+        rho = c.res_rho[off:off + cnt].astype(np.int64)
+        if B < 2 * cnt:
+            bits = np.zeros(B * 8, dtype=np.uint8)
+            bits[rho] = 1
+            masks.append(np.packbits(bits, bitorder="little"))
+            res_dir[t] = (1, n_mask)
+            n_mask += B
+        else:
+            lists.append(rho.astype(np.uint16))
+            res_dir[t] = (0, n_list)
+            n_list += cnt
+    res_list = np.concatenate(lists) if lists else np.zeros(0, dtype=np.uint16)
+    res_mask = np.concatenate(masks) if masks else np.zeros(0, dtype=np.uint8)
+    return res_dir, res_list.astype(np.uint16), res_mask.astype(np.uint8)
+
+
+def residual_expand(c: Container, res_dir, res_list, res_mask) -> np.ndarray:
+    """The inverse: the positions res_rho of every Residual entry, from the compact form."""
+    H = c.tile_k // 2
+    B = (c.tile_m * H + 7) // 8
+    out = np.zeros(len(c.res_val), dtype=np.uint16)
+    for t in range(c.tile_dir.shape[0]):
+        off, cnt = int(c.tile_dir[t, 2]), int(c.tile_dir[t, 3])
+        mode, at = int(res_dir[t, 0]), int(res_dir[t, 1])
+        if mode == 1:
+            bits = np.unpackbits(np.asarray(res_mask[at:at + B], dtype=np.uint8), bitorder="little")
+            rho = np.flatnonzero(bits)
+            if len(rho) != cnt:
+                raise ValueError("bitmap and entry count disagree")
+        else:
+            rho = np.asarray(res_list[at:at + cnt])
+        out[off:off + cnt] = rho
+    return out
+
+
+def compact_nbytes(c: Container) -> int:
+    """Size of the container with the Residual layer in its compact form."""
+    res_dir, res_list, res_mask = residual_compact(c)
+    return c.nbytes() - c.res_rho.nbytes + res_dir.nbytes + res_list.nbytes + res_mask.nbytes

@@ -308,3 +308,62 @@ def test_rejects_bad_parameters(oracle_mod):
         oracle_mod.encode(W, 4, 12)                     # tile_k not a multiple of 8
     with pytest.raises(ValueError):
         oracle_mod.encode(W, 1024, 256)                 # more than 65535 slots per tile
+
+
+# ---- compact Residual layer ---------------------------------------------------------------------
+def _bare_container(oracle_mod, tile_m, tile_k, tile_dir, res_rho):
+    z8, z16 = np.zeros(0, np.uint8), np.zeros(0, np.uint16)
+    return oracle_mod.Container(1, 1, tile_m, tile_k, 15, z16, z8, z16, z16, z8, z8, np.asarray(tile_dir, np.uint32).reshape(-1, 4),
+                                np.asarray(res_rho, np.uint16), np.zeros(len(res_rho), np.uint16))
+
+
+def test_compact_residual_golden(oracle_mod):
+    import json, os
+    g = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "residual_compact.json")))
+    c = _bare_container(oracle_mod, g["tile_m"], g["tile_k"], g["tile_dir"], g["res_rho"])
+    res_dir, res_list, res_mask = oracle_mod.residual_compact(c)
+    assert res_dir.tolist() == g["res_dir"]
+    assert res_list.tolist() == g["res_list"]
+    assert res_mask.tolist() == g["res_mask"]
+    assert oracle_mod.residual_expand(c, res_dir, res_list, res_mask).tolist() == g["res_rho"]
+
+
+def test_compact_residual_round_trip_and_size_rule(oracle_mod):
+    """Brute force on random position sets: expanding the compact form gives the positions back,
+    every tile took the smaller of its two codings, and bit b of a bitmap stands for position b."""
+    rng = np.random.default_rng(5)
+    for tile_m, tile_k in ((128, 128), (4, 32), (1, 8)):
+        slots = tile_m * tile_k // 2
+        B = (slots + 7) // 8
+        counts = [0, 1, B // 2, B // 2 + 1, slots // 3, slots]
+        tile_dir, rho = [], []
+        for n in counts:
+            tile_dir.append([0, 0, len(rho), n])
+            rho += sorted(rng.choice(slots, size=n, replace=False).tolist())
+        c = _bare_container(oracle_mod, tile_m, tile_k, tile_dir, rho)
+        res_dir, res_list, res_mask = oracle_mod.residual_compact(c)
+        assert oracle_mod.residual_expand(c, res_dir, res_list, res_mask).tolist() == rho
+        for t, n in enumerate(counts):
+            assert int(res_dir[t, 0]) == (1 if B < 2 * n else 0)
+        assert len(res_list) == sum(n for n in counts if not B < 2 * n)
+        assert len(res_mask) == B * sum(1 for n in counts if B < 2 * n)
+        # the full tile: every bit of its bitmap is set
+        t = len(counts) - 1
+        if res_dir[t, 0] == 1:
+            m = res_mask[int(res_dir[t, 1]):int(res_dir[t, 1]) + B]
+            assert int(np.unpackbits(m, bitorder="little")[:slots].sum()) == slots
+
+
+def test_compact_residual_shrinks_a_40_percent_matrix(oracle_mod):
+    """At 40 % sparsity a sixth of the non-zeros lands in the Residual layer (no tile can hold more
+    than half of its weights in value slots): the compact form must bring the container from about
+    0.81 to under 0.78 of the dense size, and leave a 50 % matrix as it is."""
+    from paper_2607_08786_b200 import workloads as wl
+    case = wl.Case(0, "s40", 512, 1024, 8, 3, 0.4, "magnitude")
+    c = oracle_mod.encode(case.make_W())
+    dense = 2 * case.M * case.K
+    assert 0.15 < c.stats["n_res"] / c.stats["nnz"] < 0.18
+    assert c.nbytes() / dense > 0.80 and oracle_mod.compact_nbytes(c) / dense < 0.78
+    assert np.array_equal(oracle_mod.residual_expand(c, *oracle_mod.residual_compact(c)), c.res_rho)
+    c50 = oracle_mod.encode(wl.Case(0, "s50", 512, 1024, 8, 3, 0.5, "magnitude").make_W())
+    assert abs(oracle_mod.compact_nbytes(c50) - c50.nbytes()) <= 8 * c50.tile_dir.shape[0]
