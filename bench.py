@@ -282,10 +282,20 @@ def run_ours(args, rank, local_rank, world):
         wt = weights[key] = Weights(tl3, c, dev, at_least=3)
         st = wt.stats
         conversion.append({"M": c.M, "K": c.K, "host_encode_s": round(wt.encode_s, 3), "device_pack_upload_s": round(wt.upload_s, 3),
-                           "canonical_bytes": st["canonical_bytes"], "device_bytes": st["device_bytes"]})
+                           "canonical_bytes": st["canonical_bytes"], "device_bytes": st["device_bytes"],
+                           # shares of the non-zeros by layer: the canonical container, and the device image that
+                           # actually streams (its chains are cut after three code words, the tails travel as
+                           # Residual entries, and its delta bytes include the zero padding of short chains)
+                           "canonical_shares": {"tc": round(st["n_tc"] / st["nnz"], 4), "sf": round(st["n_sf"] / st["nnz"], 4),
+                                                "res": round(st["n_res"] / st["nnz"], 4), "dummy": round(st["n_dummy"] / st["nnz"], 4)},
+                           "device_shares": {"tc": round(st["n_tc"] / st["nnz"], 4), "sf_coded": round(st["dev_n_sf"] / st["nnz"], 4),
+                                             "res_entries": round(st["dev_n_res"] / st["nnz"], 4),
+                                             "dummy_and_padding_bytes": round(st["dev_n_dummy"] / st["nnz"], 4)}})
         log(f"[rank {rank}] {c.M}x{c.K}: nnz {st['nnz']} TC {st['n_tc']/st['nnz']:.4f} SF {st['n_sf']/st['nnz']:.4f} "
             f"RES {st['n_res']/st['nnz']:.4f} dummies {st['n_dummy']/st['nnz']:.4f} blob {st['device_bytes']/1e6:.1f} MB "
             f"({st['device_bytes']/(2*c.M*c.K):.4f} x dense, canonical {st['canonical_bytes']/(2*c.M*c.K):.4f}) "
+            f"| device image: coded SF {st['dev_n_sf']/st['nnz']:.4f} RES entries {st['dev_n_res']/st['nnz']:.4f} "
+            f"dummy+padding bytes {st['dev_n_dummy']/st['nnz']:.4f} | "
             f"encode {wt.encode_s:.2f} s, pack+upload {wt.upload_s:.2f} s, {len(wt.blobs)} device copies")
     launches = []
     for j, c in enumerate(cases):

@@ -44,6 +44,15 @@ typedef struct {
   int64_t nnz, n_tc, n_sf, n_res, n_dummy, n_slots_unused;
   int64_t canonical_bytes;    /* sum of the nine canonical arrays                     */
   int64_t device_bytes;       /* size of the packed device blob                       */
+  int64_t canonical_bytes_compact;  /* the same with the Residual layer in its compact form        */
+  /* Layer counts of the device image, i.e. of what the kernel streams (0 for tiles other than
+   * 128 x 128).  The device image pairs and cuts the PDD chains for the banks of shared memory and
+   * sends what does not fit three code words per chain to its Residual list, so its Residual share
+   * is larger than the canonical one. */
+  int64_t dev_n_sf;           /* elements whose position is PDD-coded                               */
+  int64_t dev_n_res;          /* elements that travel as Residual entries                           */
+  int64_t dev_n_dummy;        /* delta bytes that move nothing: dummy points and chain padding      */
+  int64_t dev_pdd_bytes;      /* delta bytes in all                                                 */
 } tl3_stats_t;
 
 enum {
@@ -68,7 +77,15 @@ enum {
   TL3_PDD_BYTES = 5,   /* u8  []                t delta low nibble, r delta high nibble          */
   TL3_TILE_DIR = 6,    /* u32 [tiles][4]        pdd_off, pdd_len, res_off, res_cnt               */
   TL3_RES_RHO = 7,     /* u16 []                Residual positions                               */
-  TL3_RES_VAL = 8      /* u16 []                Residual values                                  */
+  TL3_RES_VAL = 8,     /* u16 []                Residual values                                  */
+  /* Compact form of the Residual layer (Sec. 3.2 leaves its format open: "such as CSR"), derived
+   * from TL3_RES_RHO: per tile whichever is smaller, the position list or a bitmap over the tile's
+   * tile_m * tile_k / 2 positions of W_r; values stay in TL3_RES_VAL, in ascending position order. */
+  TL3_RES_DIR = 9,     /* u32 [tiles][2]        {mode, off}: 0 = list, off indexes TL3_RES_LIST;        */
+                       /*                       1 = bitmap, off = byte offset into TL3_RES_MASK         */
+  TL3_RES_LIST = 10,   /* u16 []                positions of the list-mode tiles                         */
+  TL3_RES_MASK = 11    /* u8  []                ceil(tile_m*tile_k/16) bytes per bitmap-mode tile, bit   */
+                       /*                       rho % 8 of byte rho / 8                                  */
 };
 
 /* ---- format: host side (Sec. 3.2) ------------------------------------------------------ */

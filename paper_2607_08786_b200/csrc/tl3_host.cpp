@@ -365,9 +365,41 @@ int tl3_decode(const tl3_matrix* m, uint16_t* W_out) {
   return bad ? TL3_ERR_BAD_CONTAINER : TL3_OK;
 }
 
+// Compact form of the Residual layer: per tile the smaller of the two-byte position list and a
+// bitmap over the tile's tile_m * H positions of W_r (bit rho % 8 of byte rho / 8).  Derived from
+// res_rho on first use.
+static void ensure_compact(const tl3_matrix* m) {
+  if (m->compact_ready.load(std::memory_order_acquire)) return;
+  std::lock_guard<std::mutex> lock(m->layout_mu);
+  if (m->compact_ready.load(std::memory_order_relaxed)) return;
+  const size_t mask_bytes = (static_cast<size_t>(m->p.tile_m) * (m->p.tile_k / 2) + 7) / 8;
+  m->res_dir.assign(static_cast<size_t>(m->n_tiles) * 2, 0);
+  m->res_list.clear();
+  m->res_mask.clear();
+  for (int64_t t = 0; t < m->n_tiles; ++t) {
+    const uint32_t off = m->tile_dir[t * 4 + 2], cnt = m->tile_dir[t * 4 + 3];
+    if (mask_bytes < 2u * static_cast<size_t>(cnt)) {
+      m->res_dir[2 * t] = 1;
+      m->res_dir[2 * t + 1] = static_cast<uint32_t>(m->res_mask.size());
+      m->res_mask.resize(m->res_mask.size() + mask_bytes, 0);
+      uint8_t* bits = m->res_mask.data() + m->res_dir[2 * t + 1];
+      for (uint32_t j = off; j < off + cnt; ++j) bits[m->res_rho[j] >> 3] |= static_cast<uint8_t>(1u << (m->res_rho[j] & 7u));
+    } else {
+      m->res_dir[2 * t] = 0;
+      m->res_dir[2 * t + 1] = static_cast<uint32_t>(m->res_list.size());
+      m->res_list.insert(m->res_list.end(), m->res_rho.begin() + off, m->res_rho.begin() + off + cnt);
+    }
+  }
+  m->compact_ready.store(true, std::memory_order_release);
+}
+
 int tl3_canonical(const tl3_matrix* m, int which, const void** ptr, size_t* bytes) {
   if (!m || !ptr || !bytes) return TL3_ERR_INVALID_ARG;
+  if (which >= TL3_RES_DIR && which <= TL3_RES_MASK) ensure_compact(m);
   switch (which) {
+    case TL3_RES_DIR:    *ptr = m->res_dir.data();    *bytes = m->res_dir.size() * 4; break;
+    case TL3_RES_LIST:   *ptr = m->res_list.data();   *bytes = m->res_list.size() * 2; break;
+    case TL3_RES_MASK:   *ptr = m->res_mask.data();   *bytes = m->res_mask.size(); break;
     case TL3_TC_VALS:    *ptr = m->tc_vals.data();    *bytes = m->tc_vals.size() * 2; break;
     case TL3_TC_META:    *ptr = m->tc_meta.data();    *bytes = m->tc_meta.size(); break;
     case TL3_CHAIN_TAU0: *ptr = m->chain_tau0.data(); *bytes = m->chain_tau0.size() * 2; break;
@@ -395,6 +427,11 @@ int tl3_stats(const tl3_matrix* m, tl3_stats_t* out) {
   out->n_dummy = m->n_dummy; out->n_slots_unused = m->n_slots_unused;
   out->canonical_bytes = canonical_bytes(m);
   out->device_bytes = static_cast<int64_t>(tl3_device_bytes(m));
+  ensure_compact(m);
+  out->canonical_bytes_compact = out->canonical_bytes - static_cast<int64_t>(m->res_rho.size() * 2) +
+                                 static_cast<int64_t>(m->res_dir.size() * 4 + m->res_list.size() * 2 + m->res_mask.size());
+  out->dev_n_sf = m->dev_n_sf; out->dev_n_res = m->dev_n_res; out->dev_n_dummy = m->dev_n_dummy;
+  out->dev_pdd_bytes = m->dev_pdd_bytes;
   return TL3_OK;
 }
 

@@ -36,6 +36,13 @@ struct tl3_matrix {
   mutable uint32_t max_block_bytes = 0;
   mutable std::vector<uint32_t> dev_sizes;   // per tile: PDD bytes and Residual entries of the device image
   mutable size_t dir_offset = 0, blocks_offset = 0;
+  // layer counts of the device image (set with the layout)
+  mutable int64_t dev_n_sf = 0, dev_n_res = 0, dev_n_dummy = 0, dev_pdd_bytes = 0;
+  // compact form of the canonical Residual layer (computed on first use, under layout_mu)
+  mutable std::atomic<bool> compact_ready{false};
+  mutable std::vector<uint32_t> res_dir;
+  mutable std::vector<uint16_t> res_list;
+  mutable std::vector<uint8_t> res_mask;
 
   // last launch geometry (reporting only)
   mutable std::atomic<int> last_ctas{0}, last_stages{0}, last_smem{0};

@@ -56,7 +56,7 @@ constexpr int kChains = 128;             // four per bank
 // scattered by whichever lane is free.)
 
 struct TileCode {
-  uint32_t pdd_len = 0, res_cnt = 0;
+  uint32_t pdd_len = 0, res_cnt = 0, real_bytes = 0;        // real_bytes: delta bytes that move a value
   uint16_t vals[kSlots];                 // by pos; parked values removed, then re-parked
   uint32_t hdr[kChains];                 // by chain c (u order): u_tau0 | u_rho0 << 16
   uint8_t len[kChains];
@@ -172,6 +172,7 @@ void build_tile(const tl3_matrix* m, int64_t tm, int64_t tk, TileCode& tc) {
   const uint32_t cap = 4u * n_words;
   tc.code.clear();
   tc.res.clear();
+  tc.real_bytes = 0;
   {
     size_t i = 0;
     for (int c = 0; c < kChains; ++c) {
@@ -196,6 +197,7 @@ void build_tile(const tl3_matrix* m, int64_t tm, int64_t tk, TileCode& tc) {
           while (gt > 15) { tc.code.push_back(0x0F); gt -= 15; }     // dummy points (a zero nibble moves nothing)
           while (gr > 15) { tc.code.push_back(0xF0); gr -= 15; }
           tc.code.push_back(static_cast<uint8_t>(gt | gr << 4));
+          ++tc.real_bytes;
           n_bytes += need;
         }
         tc.vals[pos_of_u(u)] = v;
@@ -243,10 +245,24 @@ size_t plan_device_layout(const tl3_matrix* m) {
   std::lock_guard<std::mutex> lock(m->layout_mu);
   if (m->layout_ready.load(std::memory_order_relaxed)) return m->device_bytes;
   m->dev_sizes.assign(static_cast<size_t>(m->n_tiles) * 2, 0);
+  std::vector<uint32_t> real_bytes(static_cast<size_t>(m->n_tiles), 0);
   for_each_tile(m, [&](int64_t t, const TileCode& tc) {
     m->dev_sizes[2 * t] = tc.pdd_len;
     m->dev_sizes[2 * t + 1] = tc.res_cnt;
+    real_bytes[t] = tc.real_bytes;
   });
+  // layer shares of the device image (what actually streams): elements whose position is PDD-coded,
+  // elements that travel as Residual entries, and delta bytes that move nothing (dummy points and
+  // the zero bytes that pad every chain of a tile to the same number of code words)
+  m->dev_n_res = m->dev_pdd_bytes = 0;
+  int64_t real = 0;
+  for (int64_t t = 0; t < m->n_tiles; ++t) {
+    m->dev_n_res += m->dev_sizes[2 * t + 1];
+    m->dev_pdd_bytes += m->dev_sizes[2 * t];
+    real += real_bytes[t];
+  }
+  m->dev_n_sf = m->n_sf + m->n_res - m->dev_n_res;
+  m->dev_n_dummy = m->dev_pdd_bytes - real;
   size_t off = 256;
   m->dir_offset = off;
   off += static_cast<size_t>(m->n_tiles) * sizeof(DirEntry);

@@ -21,8 +21,10 @@ STATIC_SCRATCH_BYTES = 3 << 20
 
 CANONICAL = ("tc_vals", "tc_meta", "chain_tau0", "chain_rho0", "chain_len", "pdd_bytes", "tile_dir",
              "res_rho", "res_val")
+# the compact form of the Residual layer, derived from res_rho (numbered after the nine above)
+COMPACT = ("res_dir", "res_list", "res_mask")
 _CANONICAL_DTYPES = (np.uint16, np.uint8, np.uint16, np.uint16, np.uint8, np.uint8, np.uint32,
-                     np.uint16, np.uint16)
+                     np.uint16, np.uint16, np.uint32, np.uint16, np.uint8)
 
 # every symbol include/tl3.h declares
 SYMBOLS = ("tl3_encode", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_deserialize",
@@ -58,7 +60,8 @@ ACTIVATIONS = {None: 0, "none": 0, "relu": 1, "silu": 2, "gelu_tanh": 3}
 class Stats(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in
                 ("M", "K", "M_pad", "K_pad", "n_tiles", "nnz", "n_tc", "n_sf", "n_res", "n_dummy",
-                 "n_slots_unused", "canonical_bytes", "device_bytes")]
+                 "n_slots_unused", "canonical_bytes", "device_bytes", "canonical_bytes_compact",
+                 "dev_n_sf", "dev_n_res", "dev_n_dummy", "dev_pdd_bytes")]
 
     def as_dict(self) -> dict:
         return {n: int(getattr(self, n)) for n, _ in self._fields_}
@@ -195,7 +198,7 @@ class Matrix:
         return W
 
     def canonical(self, which) -> np.ndarray:
-        idx = CANONICAL.index(which) if isinstance(which, str) else int(which)
+        idx = (CANONICAL + COMPACT).index(which) if isinstance(which, str) else int(which)
         p, n = ctypes.c_void_p(), ctypes.c_size_t()
         _check(lib().tl3_canonical(self._h, idx, ctypes.byref(p), ctypes.byref(n)), "tl3_canonical")
         if n.value == 0:

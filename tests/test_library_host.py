@@ -162,6 +162,28 @@ def test_error_codes(tl3):
     assert L.tl3_strerror(-99) == b"unknown error"
 
 
+@pytest.mark.parametrize("sparsity", [0.3, 0.4, 0.5])
+def test_compact_residual_matches_the_oracle(tl3, oracle_mod, sparsity):
+    """The library's compact form of the Residual layer (list or bitmap per tile) byte for byte
+    against the oracle's, and the sizes tl3_stats reports against the arrays themselves."""
+    W = wl.Case(0, "cr", 300, 520, 8, 12, sparsity, "magnitude").make_W()
+    m = tl3.encode(W)
+    cont = oracle_mod.encode(W)
+    res_dir, res_list, res_mask = oracle_mod.residual_compact(cont)
+    assert np.array_equal(m.canonical("res_dir").reshape(-1, 2), res_dir)
+    assert np.array_equal(m.canonical("res_list"), res_list)
+    assert np.array_equal(m.canonical("res_mask"), res_mask)
+    st = m.stats()
+    assert st["canonical_bytes"] == cont.nbytes()
+    assert st["canonical_bytes_compact"] == oracle_mod.compact_nbytes(cont)
+    if sparsity < 0.5:
+        assert (res_dir[:, 0] == 1).any()
+    # the device image's own layer counts add up to the surplus elements of the matrix; its
+    # Residual list also takes what the three code words of a chain cannot hold
+    assert st["dev_n_sf"] + st["dev_n_res"] == st["n_sf"] + st["n_res"]
+    assert st["dev_n_res"] >= st["n_res"] and 0 <= st["dev_n_dummy"] <= st["dev_pdd_bytes"]
+
+
 def test_launch_tuning_round_trip(tl3):
     L = tl3.lib()
     assert tl3.get_tuning() == {"decode_before_x": 4}
