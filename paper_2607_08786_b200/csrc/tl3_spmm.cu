@@ -116,8 +116,8 @@ enum : uint32_t { kOptSplitX = 1u };
 static long long* g_timing_buffer = nullptr;
 static int g_timing_launch = 0;
 __device__ __forceinline__ long long clock_now() { long long c; asm volatile("mov.u64 %0, %%clock64;" : "=l"(c) :: "memory"); return c; }
-#define TL3_GT(k) { if (a.timing) a.timing[blockIdx.x * 16 + (k)] = clock_now(); }
-#define TL3_GV(k, v) { if (a.timing) a.timing[blockIdx.x * 16 + (k)] = static_cast<long long>(v); }
+#define TL3_GT(k) { if (a.timing) a.timing[blockIdx.x * 32 + (k)] = clock_now(); }
+#define TL3_GV(k, v) { if (a.timing) a.timing[blockIdx.x * 32 + (k)] = static_cast<long long>(v); }
 #else
 #define TL3_GT(k) {}
 #define TL3_GV(k, v) {}
@@ -424,6 +424,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     mbar_init(bar_tail, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    TL3_GT(16)
   }
   // the producer's first directory entries and the X tensor map: start the (cold) global fetches
   // before the set-up barrier
@@ -435,10 +436,12 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   if (warp == kAllocWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (lane == 0) { TL3_GT(19) }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (tid == 0) { TL3_GT(17) }
   const uint32_t tmem_base = *tmem_slot;
   const WaitCtx wctx{abort_flag, a.status};
   pdl_launch_dependents();
@@ -465,6 +468,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       if (base == 0) {
         for (int j = 0; j < pre; ++j) {                          // S <= 8 < 32: all in this batch
           const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.x, j), bytes = __shfl_sync(0xFFFFFFFFu, mine.y, j);
+          if (lane == 0 && j == 0 && off16 != 0xFFFFFFFFu) { TL3_GT(18) }
           const uint8_t* src = a.blob + static_cast<size_t>(off16) * 16;
           const uint32_t st = smem_base + static_cast<uint32_t>(j) * a.stage_stride, full = bar_full + 8 * j;
           if (elect_one()) {
@@ -1100,7 +1104,7 @@ static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, 
   const long long tiles_per_cta = (total + grid - 1) / grid;
   args.opts = (dbx < 0 || tiles_per_cta <= dbx) ? kOptSplitX : 0u;
 #ifdef TL3_CTA_STAMPS
-  args.timing = g_timing_buffer ? g_timing_buffer + static_cast<long long>(g_timing_launch++ % 64) * 148 * 16 : nullptr;
+  args.timing = g_timing_buffer ? g_timing_buffer + static_cast<long long>(g_timing_launch++ % 64) * 148 * 32 : nullptr;
 #else
   args.timing = nullptr;
 #endif
@@ -1283,7 +1287,7 @@ int tl3_selftest_bounded_wait(void* workspace, void* stream) {
 }
 
 #ifdef TL3_CTA_STAMPS
-void tl3_debug_set_timing_buffer(long long* device_ptr) { tl3::g_timing_buffer = device_ptr; tl3::g_timing_launch = 0; }   // 64 x 148 x 16 int64
+void tl3_debug_set_timing_buffer(long long* device_ptr) { tl3::g_timing_buffer = device_ptr; tl3::g_timing_launch = 0; }   // 64 x 148 x 32 int64
 #endif
 
 }  // extern "C"
