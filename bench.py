@@ -218,6 +218,15 @@ class Weights:
             self.dense = [d0] + [d0.clone() for _ in range(min(len(self.blobs), _copies_for(W.nbytes, at_least)) - 1)]
         self.W = W
         self.stats = self.m.stats()
+        # the same container built by the CUDA encoder (window classification, scans, pairing, chain
+        # emission on the GPU; the copy of the arrays back to the host is inside the time)
+        self.device_encode_s, self.device_encode_identical = None, None
+        if dense:
+            t0 = time.perf_counter()
+            md = tl3.Matrix.encode_on_device(self.dense[0])
+            self.device_encode_s = time.perf_counter() - t0
+            self.device_encode_identical = all(np.array_equal(md.canonical(n), self.m.canonical(n)) for n in ("pdd_bytes", "tile_dir", "res_rho", "chain_len"))
+            md.close()
 
     def spmm(self, i, X, Y, ws, stream=None):
         self.m.bind(self.blobs[i % len(self.blobs)])
@@ -282,6 +291,7 @@ def run_ours(args, rank, local_rank, world):
         wt = weights[key] = Weights(tl3, c, dev, at_least=3)
         st = wt.stats
         conversion.append({"M": c.M, "K": c.K, "host_encode_s": round(wt.encode_s, 3), "device_pack_upload_s": round(wt.upload_s, 3),
+                           "gpu_encode_s": round(wt.device_encode_s, 3), "gpu_encode_identical": wt.device_encode_identical,
                            "canonical_bytes": st["canonical_bytes"], "device_bytes": st["device_bytes"],
                            # shares of the non-zeros by layer: the canonical container, and the device image that
                            # actually streams (its chains are cut after three code words, the tails travel as

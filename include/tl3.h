@@ -95,6 +95,17 @@ enum {
  * caller releases with tl3_free().  Errors: INVALID_ARG (NULL, M or K <= 0, bad params). */
 int tl3_encode(const uint16_t* W, int64_t M, int64_t K, const tl3_params* params, tl3_matrix** out);
 
+/* The same conversion on the GPU (the paper converts on the CPU and quotes 41-93 s per model,
+ * Sec. 5.3): window classification, ordered lists of surplus weights and empty slots by prefix
+ * scans, pairing and chain emission run as CUDA kernels, one CTA per 128 x 128 tile; the result is
+ * the same canonical container, byte for byte, in a new handle with host copies of the arrays
+ * (tl3_decode, tl3_upload, tl3_serialize ... work on it as on any other).
+ *   dW: device, fp16 bits, row-major M x K, leading dimension ldw >= K, already masked.
+ *   Tile 128 x 128, maxd 15 only.  The call allocates and frees device scratch of about the size
+ *   of the container (cudaMalloc), runs on `stream` and waits for it.
+ * Errors: INVALID_ARG, UNSUPPORTED (more than 4 GiB of PDD bytes), CUDA, NO_MEMORY. */
+int tl3_encode_device(const void* dW, int64_t M, int64_t K, int64_t ldw, void* stream, tl3_matrix** out);
+
 /* Decode back to dense: Algorithm 1 run on the host, then the 2:4 expansion and the Residual
  * entries.  W_out: host, M*K uint16_t, caller-owned, fully overwritten.  The result equals the
  * encoder's input bit for bit (with -0.0 read as +0.0).  Errors: BAD_CONTAINER. */

@@ -634,3 +634,76 @@ def test_row_sharded_matrix_on_one_rank(tl3, oracle_mod):
     Y = sh.matmul(device_X(X))
     torch.cuda.synchronize()
     check(oracle_mod, W, X, Y.cpu().numpy())
+
+
+def _device_encode_matches(tl3, oracle_mod, W, ld=None):
+    import torch
+    M, K = W.shape
+    buf = torch.zeros((M, ld or K), dtype=torch.float16, device="cuda")
+    buf[:, :K] = torch.from_numpy(W)
+    m = tl3.Matrix.encode_on_device(buf[:, :K])
+    cont = oracle_mod.encode(W)
+    for name in tl3.CANONICAL:
+        assert np.array_equal(m.canonical(name), getattr(cont, name).ravel()), name
+    st = m.stats()
+    for key in ("nnz", "n_tc", "n_sf", "n_res", "n_dummy", "n_slots_unused"):
+        assert st[key] == cont.stats[key], key
+    assert np.array_equal(m.decode(), np.where((W.view(np.uint16) & 0x7FFF) == 0, 0, W.view(np.uint16)))
+    return m
+
+
+@pytest.mark.parametrize("shape,sparsity,kind", [((1024, 1024), 0.5, "bernoulli"), ((640, 896), 0.5, "magnitude"),
+                                                 ((1000, 1096), 0.4, "magnitude"), ((130, 260), 0.6, "magnitude"),
+                                                 ((384, 512), 0.7, "magnitude"), ((256, 384), 0.0, "bernoulli"),
+                                                 ((1, 8), 0.5, "bernoulli"), ((2048, 4096), 0.5, "wanda")])
+def test_gpu_encoder_is_byte_identical_to_the_oracle(tl3, oracle_mod, shape, sparsity, kind):
+    """The container built by the CUDA encoder (window classification, ordered lists by prefix
+    scans, pairing, chain emission, Residual) against the oracle's, array by array and count by
+    count, on aligned and ragged shapes and on the dense and sparse side of 50 %."""
+    W = wl.Case(0, "ge", shape[0], shape[1], 8, 70 + shape[0], sparsity, kind).make_W()
+    _device_encode_matches(tl3, oracle_mod, W)
+
+
+def test_gpu_encoder_on_hand_built_patterns(tl3, oracle_mod):
+    """Dummy points, a chain cut after 255 bytes, cross-row parking, -0.0, a strided source, and the
+    product computed from the device-encoded handle."""
+    import torch
+    from special_cases import clustered_surplus_tile
+    rng = np.random.default_rng(3)
+    # top half of every tile dense, bottom half empty: every surplus weight is parked in another row
+    W = np.zeros((256, 256), dtype=np.float16)
+    W[:64] = (rng.standard_normal((64, 256)) * 0.05 + 0.2).astype(np.float16)
+    W[128:192] = (rng.standard_normal((64, 256)) * 0.05 + 0.2).astype(np.float16)
+    _device_encode_matches(tl3, oracle_mod, W)
+    # surplus weights in row 0 only, empty slots spread over the whole tile: long spans of dummy
+    # points, and the row's chain runs into the 255-byte limit
+    W = (rng.standard_normal((128, 128)) * 0.05 + 0.3).astype(np.float16)
+    W[1:, 2::4] = 0
+    W[1:, 3::4] = 0
+    W[1::2, 1::4] = 0
+    m = _device_encode_matches(tl3, oracle_mod, W)
+    assert m.stats()["n_dummy"] > 0
+    # row 0 dense (64 surplus weights), the other rows exactly 2:4 with one empty slot every 115
+    # slots: eight dummy bytes per pair, so the chain of row 0 is cut at 255 bytes and the rest of the
+    # row goes to the Residual layer
+    W = np.zeros((128, 128), dtype=np.float16)
+    base = (rng.standard_normal((128, 128)) * 0.05 + 0.3).astype(np.float16)
+    W[0] = base[0]
+    W[1:, 0::4] = base[1:, 0::4]
+    W[1:, 1::4] = base[1:, 1::4]
+    for k in range(70):
+        tau = 64 + k * 115
+        W[tau // 64, 4 * ((tau % 64) // 2) + (tau & 1)] = 0
+    m = _device_encode_matches(tl3, oracle_mod, W)
+    assert m.stats()["n_res"] == 32 and m.canonical("chain_len")[0] == 248
+    _device_encode_matches(tl3, oracle_mod, clustered_surplus_tile())
+    W = wl.Case(0, "neg0", 300, 520, 8, 4, 0.5, "magnitude").make_W()
+    W.view(np.uint16)[W == 0] = 0x8000                                  # pruned weights as -0.0
+    _device_encode_matches(tl3, oracle_mod, W)
+    case = wl.Case(0, "ld", 512, 640, 16, 8, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    m = _device_encode_matches(tl3, oracle_mod, W, ld=648)
+    m.upload()
+    Y = m.spmm(device_X(X))
+    torch.cuda.synchronize()
+    check(oracle_mod, W, X, Y.cpu().numpy())
