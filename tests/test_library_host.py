@@ -158,6 +158,14 @@ def test_error_codes(tl3):
     assert L.tl3_spmm(m._h, 16, 8, 16, 8, 8, 256, None) == tl3.ERR_NOT_UPLOADED
     assert L.tl3_spmm(None, None, 8, None, 8, 8, None, None) == tl3.ERR_INVALID_ARG
     assert L.tl3_workspace_bytes(m._h, 4097) == 0 and L.tl3_workspace_bytes(m._h, 0) == 0
+    # argument checks of the entry points that need a device come before any CUDA call
+    hd = ctypes.c_void_p()
+    assert L.tl3_encode_device(None, 8, 8, 8, None, ctypes.byref(hd)) == tl3.ERR_INVALID_ARG
+    assert L.tl3_encode_device(256, 8, 16, 8, None, ctypes.byref(hd)) == tl3.ERR_INVALID_ARG      # ldw < K
+    assert L.tl3_bind(None, 256) == tl3.ERR_INVALID_ARG
+    assert L.tl3_bind(m._h, 256) == tl3.ERR_UNSUPPORTED                                            # 8 x 16 tiles
+    m128 = tl3.encode(np.zeros((8, 16), dtype=np.float16))
+    assert L.tl3_bind(m128._h, 260) == tl3.ERR_INVALID_ARG                                         # not 256-byte aligned
     assert b"invalid" in L.tl3_strerror(tl3.ERR_INVALID_ARG)
     assert L.tl3_strerror(-99) == b"unknown error"
 
