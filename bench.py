@@ -416,18 +416,38 @@ def run_ours(args, rank, local_rank, world):
         for s in e2e_streams:
             s.synchronize()
 
-    for _ in range(3):
-        step_e2e()
-    e2e_blocks = []
-    for _ in range(3):
-        dist.barrier()
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        for _ in range(args.steps):
-            step_e2e()
-        torch.cuda.synchronize()
-        e2e_blocks.append(dist.max_over_ranks((time.perf_counter() - t0) / args.steps, device=dev))
-    e2e_s = float(np.median(e2e_blocks))
+    def timed_e2e(step_fn):
+        for _ in range(3):
+            step_fn()
+        out = []
+        for _ in range(3):
+            dist.barrier()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(args.steps):
+                step_fn()
+            torch.cuda.synchronize()
+            out.append(dist.max_over_ranks((time.perf_counter() - t0) / args.steps, device=dev))
+        return float(np.median(out)), out
+
+    e2e_eager_s, _ = timed_e2e(step_e2e)
+    # The same nine calls (copy in, kernel, copy out each, three streams) captured once as a CUDA
+    # graph -- tl3_spmm_host_async only enqueues, so a caller can do that -- and replayed per step; the
+    # step ends when the host has waited for the stream, i.e. when every Y is in host memory.
+    def e2e_call(st, L, bufs):
+        Xp, Yp, dX, dY = bufs
+        L["wt"].m.bind(L["wt"].blobs[L["copy"]])
+        L["wt"].m.spmm_host_async(Xp, Yp, dX, dY, L["ws"], stream=st)
+
+    e2e_graph = _capture(forked([(lambda st, L=L, b=b: e2e_call(st, L, b)) for L, b in zip(launches, e2e_bufs)]))
+
+    def step_e2e_graph():
+        e2e_graph.replay()
+        torch.cuda.current_stream().synchronize()
+
+    for (Xp, Yp, dX, dY) in e2e_bufs:
+        Yp[:] = 0
+    e2e_s, e2e_blocks = timed_e2e(step_e2e_graph)
     e2e_value = total_bytes / e2e_s / 1e9
     h2d = sum(L["Xh"].nbytes for L in launches)
     d2h = sum(L["case"].M * L["case"].N * 2 for L in launches)
@@ -490,7 +510,10 @@ def run_ours(args, rank, local_rank, world):
         "clocks": clocks,
         "gpu_launches": len(launches_info) * args.steps * BLOCKS,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_s * 1e3, "blocks_ms_per_step": [round(b * 1e3, 4) for b in e2e_blocks]},
+                "ms_per_step": e2e_s * 1e3, "blocks_ms_per_step": [round(b * 1e3, 4) for b in e2e_blocks],
+                "how": "tl3_spmm_host_async x 9 on three streams captured as one CUDA graph; per step: replay, then wait for the stream "
+                       "(every Y in pinned host memory); host wall clock",
+                "eager_ms_per_step": e2e_eager_s * 1e3},
         "roofline": {"bound": "hbm", "achieved": step_bytes / (ms_step * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
                      "frac": step_bytes / (ms_step * 1e-3) / 1e9 / peak,
                      "peak_kind": f"of {peak_kind}", "frac_nominal_8tbs": step_bytes / (ms_step * 1e-3) / 1e9 / 8000.0,
