@@ -220,12 +220,20 @@ class Weights:
         self.stats = self.m.stats()
         # the same container built by the CUDA encoder (window classification, scans, pairing, chain
         # emission on the GPU; the copy of the arrays back to the host is inside the time)
-        self.device_encode_s, self.device_encode_identical = None, None
+        self.device_encode_s, self.device_encode_identical, self.device_pack_s, self.device_pack_identical = None, None, None, None
         if dense:
             t0 = time.perf_counter()
             md = tl3.Matrix.encode_on_device(self.dense[0])
             self.device_encode_s = time.perf_counter() - t0
             self.device_encode_identical = all(np.array_equal(md.canonical(n), self.m.canonical(n)) for n in ("pdd_bytes", "tile_dir", "res_rho", "chain_len"))
+            # ... and packed for the kernel by the CUDA packer (layout pass, blob pass, the copy of the
+            # canonical arrays to the device inside the time)
+            t0 = time.perf_counter()
+            blob_d = md.upload_packed_on_device(device=dev)
+            torch.cuda.synchronize()
+            self.device_pack_s = time.perf_counter() - t0
+            self.device_pack_identical = bool(torch.equal(blob_d, first))
+            del blob_d
             md.close()
 
     def spmm(self, i, X, Y, ws, stream=None):
@@ -292,6 +300,7 @@ def run_ours(args, rank, local_rank, world):
         st = wt.stats
         conversion.append({"M": c.M, "K": c.K, "host_encode_s": round(wt.encode_s, 3), "device_pack_upload_s": round(wt.upload_s, 3),
                            "gpu_encode_s": round(wt.device_encode_s, 3), "gpu_encode_identical": wt.device_encode_identical,
+                           "gpu_pack_s": round(wt.device_pack_s, 3), "gpu_pack_identical": wt.device_pack_identical,
                            "canonical_bytes": st["canonical_bytes"], "device_bytes": st["device_bytes"],
                            # shares of the non-zeros by layer: the canonical container, and the device image that
                            # actually streams (its chains are cut after three code words, the tails travel as

@@ -146,6 +146,17 @@ int tl3_pack(const tl3_matrix* m, void* host_buf, size_t bytes);
  * Errors: UNSUPPORTED (tile shape other than 128 x 128), INVALID_ARG, CUDA. */
 int tl3_upload(tl3_matrix* m, void* dptr, void* stream);
 
+/* The device packer on the GPU.  tl3_plan_device() computes the layout of the device image with a
+ * CUDA kernel (afterwards tl3_device_bytes() returns at once instead of running the host packer's
+ * first pass), tl3_upload_device() writes the blob into dptr with a second pass of the same
+ * kernel: the same bytes as tl3_pack() / tl3_upload().  Both copy the canonical arrays to the
+ * device first (one cudaMalloc of the container's size, shared between the two calls, released
+ * by tl3_upload_device or tl3_free), run on `stream` and wait for it.
+ *   dptr: device, >= tl3_device_bytes(), 256-byte aligned; bound to the handle on success.
+ * Errors: INVALID_ARG, UNSUPPORTED (tile shape other than 128 x 128), CUDA, NO_MEMORY. */
+int tl3_plan_device(tl3_matrix* m, void* stream);
+int tl3_upload_device(tl3_matrix* m, void* dptr, void* stream);
+
 /* Bind a device buffer that already holds the packed blob -- the bytes of tl3_pack() copied to the
  * device by the caller, or a device-side copy of a blob that tl3_upload() wrote -- to the handle:
  * later tl3_spmm* calls read the weights from there.  dptr: device, >= tl3_device_bytes(),

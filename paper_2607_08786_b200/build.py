@@ -8,7 +8,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libtl3.so")
-SOURCES = ("tl3_host.cpp", "tl3_pack.cpp", "tl3_spmm.cu", "tl3_encode.cu")
+SOURCES = ("tl3_host.cpp", "tl3_pack.cpp", "tl3_spmm.cu", "tl3_encode.cu", "tl3_pack_device.cu")
 HEADERS = (os.path.join(CSRC, "tl3_internal.h"), os.path.join(ROOT, "include", "tl3.h"))
 
 

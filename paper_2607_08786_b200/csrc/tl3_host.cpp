@@ -515,7 +515,10 @@ int tl3_deserialize(const void* buf, size_t bytes, tl3_matrix** out) {
   return TL3_OK;
 }
 
-void tl3_free(tl3_matrix* m) { delete m; }
+void tl3_free(tl3_matrix* m) {
+  if (m && m->device_canon && m->release_device_canon) m->release_device_canon(m->device_canon);
+  delete m;
+}
 
 const char* tl3_strerror(int code) {
   switch (code) {

@@ -27,6 +27,10 @@ struct tl3_matrix {
 
   // device binding (filled by tl3_upload)
   void* dptr = nullptr;
+  // device copies of the canonical arrays between tl3_plan_device and tl3_upload_device (one
+  // cudaMalloc, released by tl3_upload_device or tl3_free through `release_device_canon`)
+  void* device_canon = nullptr;
+  void (*release_device_canon)(void*) = nullptr;
   // Layout of the device image, computed on first use (tl3_device_bytes, tl3_pack, tl3_upload,
   // tl3_stats) under `layout_mu`, so that calls that take a const handle may share it between
   // threads; `layout_ready` is set last.
@@ -85,6 +89,8 @@ struct DirEntry {
 
 size_t plan_device_layout(const tl3_matrix* m);           // fills device_bytes, offsets, max block (once, thread-safe)
 void pack_device_blob(const tl3_matrix* m, uint8_t* out); // out: device_bytes bytes, host
+void set_device_layout(const tl3_matrix* m, const uint32_t* sizes);   // layout from per-tile sizes computed on the GPU
+void blob_header_and_offsets(const tl3_matrix* m, uint8_t* header256, std::vector<unsigned long long>* block_off);
 
 void set_cuda_error(int e);
 

@@ -239,18 +239,9 @@ void for_each_tile(const tl3_matrix* m, F&& f) {
 
 }  // namespace
 
-size_t plan_device_layout(const tl3_matrix* m) {
-  if (m->p.tile_m != kTileM || m->p.tile_k != kTileK) return 0;   // the device image exists for 128 x 128 tiles only
-  if (m->layout_ready.load(std::memory_order_acquire)) return m->device_bytes;
-  std::lock_guard<std::mutex> lock(m->layout_mu);
-  if (m->layout_ready.load(std::memory_order_relaxed)) return m->device_bytes;
-  m->dev_sizes.assign(static_cast<size_t>(m->n_tiles) * 2, 0);
-  std::vector<uint32_t> real_bytes(static_cast<size_t>(m->n_tiles), 0);
-  for_each_tile(m, [&](int64_t t, const TileCode& tc) {
-    m->dev_sizes[2 * t] = tc.pdd_len;
-    m->dev_sizes[2 * t + 1] = tc.res_cnt;
-    real_bytes[t] = tc.real_bytes;
-  });
+// From the per-tile sizes to the layout of the blob and the layer counts of the device image.
+// Caller holds layout_mu.
+static void finish_device_layout(const tl3_matrix* m, const std::vector<uint32_t>& real_bytes) {
   // layer shares of the device image (what actually streams): elements whose position is PDD-coded,
   // elements that travel as Residual entries, and delta bytes that move nothing (dummy points and
   // the zero bytes that pad every chain of a tile to the same number of code words)
@@ -277,7 +268,51 @@ size_t plan_device_layout(const tl3_matrix* m) {
   m->max_block_bytes = max_block;
   m->device_bytes = (off + 255) / 256 * 256;
   m->layout_ready.store(true, std::memory_order_release);
+}
+
+size_t plan_device_layout(const tl3_matrix* m) {
+  if (m->p.tile_m != kTileM || m->p.tile_k != kTileK) return 0;   // the device image exists for 128 x 128 tiles only
+  if (m->layout_ready.load(std::memory_order_acquire)) return m->device_bytes;
+  std::lock_guard<std::mutex> lock(m->layout_mu);
+  if (m->layout_ready.load(std::memory_order_relaxed)) return m->device_bytes;
+  m->dev_sizes.assign(static_cast<size_t>(m->n_tiles) * 2, 0);
+  std::vector<uint32_t> real_bytes(static_cast<size_t>(m->n_tiles), 0);
+  for_each_tile(m, [&](int64_t t, const TileCode& tc) {
+    m->dev_sizes[2 * t] = tc.pdd_len;
+    m->dev_sizes[2 * t + 1] = tc.res_cnt;
+    real_bytes[t] = tc.real_bytes;
+  });
+  finish_device_layout(m, real_bytes);
   return m->device_bytes;
+}
+
+// The same layout from sizes that were computed elsewhere (the pack kernel's count pass):
+// sizes[3 t] = PDD bytes, [3 t + 1] = Residual entries, [3 t + 2] = delta bytes that move a value.
+void set_device_layout(const tl3_matrix* m, const uint32_t* sizes) {
+  std::lock_guard<std::mutex> lock(m->layout_mu);
+  if (m->layout_ready.load(std::memory_order_relaxed)) return;
+  m->dev_sizes.assign(static_cast<size_t>(m->n_tiles) * 2, 0);
+  std::vector<uint32_t> real_bytes(static_cast<size_t>(m->n_tiles), 0);
+  for (int64_t t = 0; t < m->n_tiles; ++t) {
+    m->dev_sizes[2 * t] = sizes[3 * t];
+    m->dev_sizes[2 * t + 1] = sizes[3 * t + 1];
+    real_bytes[t] = sizes[3 * t + 2];
+  }
+  finish_device_layout(m, real_bytes);
+}
+
+// Offsets of the tile blocks and the 256-byte header of a blob (what pack_device_blob writes first).
+void blob_header_and_offsets(const tl3_matrix* m, uint8_t* header256, std::vector<unsigned long long>* block_off) {
+  std::memset(header256, 0, 256);
+  struct { uint32_t magic, version; int64_t M, K, M_pad, K_pad, n_tiles; uint64_t dir_off, blocks_off; uint32_t max_block; } hdr{
+      0x33334C54u, 2, m->M, m->K, m->M_pad, m->K_pad, m->n_tiles, m->dir_offset, m->blocks_offset, m->max_block_bytes};
+  std::memcpy(header256, &hdr, sizeof(hdr));
+  block_off->resize(static_cast<size_t>(m->n_tiles));
+  size_t off = m->blocks_offset;
+  for (int64_t t = 0; t < m->n_tiles; ++t) {
+    (*block_off)[t] = off;
+    off += align_up(block_bytes(m->dev_sizes[2 * t], m->dev_sizes[2 * t + 1]), kBlockAlign);
+  }
 }
 
 void pack_device_blob(const tl3_matrix* m, uint8_t* out) {

@@ -28,7 +28,7 @@ _CANONICAL_DTYPES = (np.uint16, np.uint8, np.uint16, np.uint16, np.uint8, np.uin
 
 # every symbol include/tl3.h declares
 SYMBOLS = ("tl3_encode", "tl3_encode_device", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_deserialize",
-           "tl3_free", "tl3_device_bytes", "tl3_pack", "tl3_upload", "tl3_bind", "tl3_workspace_bytes", "tl3_workspace_init",
+           "tl3_free", "tl3_device_bytes", "tl3_pack", "tl3_upload", "tl3_bind", "tl3_plan_device", "tl3_upload_device", "tl3_workspace_bytes", "tl3_workspace_init",
            "tl3_spmm", "tl3_spmm_ex", "tl3_spmm_nt", "tl3_spmm_host", "tl3_spmm_host_async", "tl3_spmm_static_scratch", "tl3_static_scratch_status", "tl3_status", "tl3_status_word", "tl3_selftest_bounded_wait", "tl3_last_launch", "tl3_strerror",
            "tl3_last_cuda_error", "tl3_get_tuning", "tl3_set_tuning")
 
@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
         L.tl3_pack.argtypes = [vp, vp, sz]
         L.tl3_upload.argtypes = [vp, vp, vp]
         L.tl3_bind.argtypes = [vp, vp]
+        L.tl3_plan_device.argtypes = [vp, vp]
+        L.tl3_upload_device.argtypes = [vp, vp, vp]
         L.tl3_workspace_bytes.argtypes = [vp, ci]
         L.tl3_workspace_bytes.restype = sz
         L.tl3_workspace_init.argtypes = [vp, sz, vp]
@@ -240,6 +242,15 @@ class Matrix:
         import torch
         blob = torch.empty(self.device_bytes(), dtype=torch.uint8, device=device)
         _check(lib().tl3_upload(self._h, blob.data_ptr(), _stream_ptr(stream)), "tl3_upload")
+        self._blob = blob
+        return blob
+
+    def upload_packed_on_device(self, device="cuda", stream=None):
+        """As :meth:`upload`, with the device packer running on the GPU (same bytes)."""
+        import torch
+        _check(lib().tl3_plan_device(self._h, _stream_ptr(stream)), "tl3_plan_device")
+        blob = torch.empty(self.device_bytes(), dtype=torch.uint8, device=device)
+        _check(lib().tl3_upload_device(self._h, blob.data_ptr(), _stream_ptr(stream)), "tl3_upload_device")
         self._blob = blob
         return blob
 

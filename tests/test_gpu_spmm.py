@@ -707,3 +707,59 @@ def test_gpu_encoder_on_hand_built_patterns(tl3, oracle_mod):
     Y = m.spmm(device_X(X))
     torch.cuda.synchronize()
     check(oracle_mod, W, X, Y.cpu().numpy())
+
+
+def _gpu_pack_matches(tl3, W):
+    """The blob written by the CUDA packer against the host packer's, byte for byte, with the layout
+    computed on the GPU (fresh handle) and on the host (second handle)."""
+    import torch
+    ref = tl3.encode(W)
+    want = ref.pack()
+    st_ref = ref.stats()
+    for host_plan_first in (False, True):
+        m = tl3.encode(W)
+        if host_plan_first:
+            assert m.device_bytes() == want.size
+        blob = m.upload_packed_on_device()
+        torch.cuda.synchronize()
+        got = blob.cpu().numpy()
+        assert got.size == want.size
+        assert np.array_equal(got, want), f"first difference at byte {int(np.flatnonzero(got != want)[0])}"
+        st = m.stats()
+        for key in ("device_bytes", "dev_n_sf", "dev_n_res", "dev_n_dummy", "dev_pdd_bytes"):
+            assert st[key] == st_ref[key], key
+    return m
+
+
+@pytest.mark.parametrize("shape,sparsity,kind", [((1024, 1024), 0.5, "bernoulli"), ((640, 896), 0.5, "magnitude"),
+                                                 ((1000, 1096), 0.4, "magnitude"), ((384, 512), 0.6, "magnitude"),
+                                                 ((384, 512), 0.7, "magnitude"), ((256, 384), 0.0, "bernoulli"),
+                                                 ((128, 128), 1.0, "bernoulli"), ((2048, 4096), 0.5, "wanda")])
+def test_gpu_packer_is_byte_identical_to_the_host_packer(tl3, shape, sparsity, kind):
+    W = wl.Case(0, "gp", shape[0], shape[1], 8, 90 + shape[0], sparsity, kind).make_W()
+    _gpu_pack_matches(tl3, W)
+
+
+def test_gpu_packer_on_adversarial_patterns_and_end_to_end(tl3, oracle_mod):
+    """Abruptly changing densities (the packer's proportional selection, equal-count chains and the
+    cut after three code words), the clustered tile whose chains overflow, and a product computed
+    from a matrix that never met the host encoder or the host packer."""
+    import torch
+    from special_cases import clustered_surplus_tile
+    for seed in range(4):
+        rng = np.random.default_rng([77, seed])
+        M, K = 256, 384
+        dens_r = rng.choice([0.0, 0.1, 0.5, 0.9, 1.0], size=M // 32).repeat(32)
+        dens_c = rng.choice([0.0, 0.25, 0.5, 0.75, 1.0], size=K // 64).repeat(64)
+        p = np.clip(0.5 * (dens_r[:, None] + dens_c[None, :]) + rng.choice([-0.3, 0.0, 0.3]), 0, 1)
+        W = np.where(rng.random((M, K)) < p, (rng.standard_normal((M, K)) * 0.05).astype(np.float16), np.float16(0))
+        W[(W.view(np.uint16) & 0x7FFF) == 0] = 0
+        _gpu_pack_matches(tl3, W)
+    _gpu_pack_matches(tl3, clustered_surplus_tile())
+    case = wl.Case(0, "gpu_only", 1536, 2048, 16, 61, 0.5, "magnitude")
+    W, X = case.make_W(), case.make_X()
+    m = tl3.Matrix.encode_on_device(torch.from_numpy(W).cuda())
+    m.upload_packed_on_device()
+    Y = m.spmm(device_X(X))
+    torch.cuda.synchronize()
+    check(oracle_mod, W, X, Y.cpu().numpy())
