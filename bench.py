@@ -222,19 +222,23 @@ class Weights:
         # emission on the GPU; the copy of the arrays back to the host is inside the time)
         self.device_encode_s, self.device_encode_identical, self.device_pack_s, self.device_pack_identical = None, None, None, None
         if dense:
-            t0 = time.perf_counter()
-            md = tl3.Matrix.encode_on_device(self.dense[0])
-            self.device_encode_s = time.perf_counter() - t0
-            self.device_encode_identical = all(np.array_equal(md.canonical(n), self.m.canonical(n)) for n in ("pdd_bytes", "tile_dir", "res_rho", "chain_len"))
-            # ... and packed for the kernel by the CUDA packer (layout pass, blob pass, the copy of the
-            # canonical arrays to the device inside the time)
-            t0 = time.perf_counter()
-            blob_d = md.upload_packed_on_device(device=dev)
-            torch.cuda.synchronize()
-            self.device_pack_s = time.perf_counter() - t0
-            self.device_pack_identical = bool(torch.equal(blob_d, first))
-            del blob_d
-            md.close()
+            enc, pack = [], []
+            for _ in range(2):                               # best of two: the first call of a kind pays for the module load
+                t0 = time.perf_counter()
+                md = tl3.Matrix.encode_on_device(self.dense[0])
+                enc.append(time.perf_counter() - t0)
+                self.device_encode_identical = all(np.array_equal(md.canonical(n), self.m.canonical(n))
+                                                   for n in ("pdd_bytes", "tile_dir", "res_rho", "chain_len"))
+                # ... and packed for the kernel by the CUDA packer (layout pass, blob pass, the copy of
+                # the canonical arrays to the device inside the time)
+                t0 = time.perf_counter()
+                blob_d = md.upload_packed_on_device(device=dev)
+                torch.cuda.synchronize()
+                pack.append(time.perf_counter() - t0)
+                self.device_pack_identical = bool(torch.equal(blob_d, first))
+                del blob_d
+                md.close()
+            self.device_encode_s, self.device_pack_s = min(enc), min(pack)
 
     def spmm(self, i, X, Y, ws, stream=None):
         self.m.bind(self.blobs[i % len(self.blobs)])
