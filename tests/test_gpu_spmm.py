@@ -763,3 +763,46 @@ def test_gpu_packer_on_adversarial_patterns_and_end_to_end(tl3, oracle_mod):
     Y = m.spmm(device_X(X))
     torch.cuda.synchronize()
     check(oracle_mod, W, X, Y.cpu().numpy())
+
+
+def test_random_shapes_through_every_gpu_route(tl3, oracle_mod):
+    """Seeded random shapes, sparsities from dense to 99 %, patchy row densities and padded leading
+    dimensions: the CUDA encoder's container and the CUDA packer's blob against the host library's
+    (itself pinned to the oracle byte for byte), then the product -- plain, transposed, and with a
+    bias and an activation -- against the oracle's fp64 result."""
+    import torch
+    rng = np.random.default_rng(20260708)
+    for it in range(24):
+        M = int(rng.integers(1, 12)) * 128 + int(rng.choice([0, 0, 1, 37, 64, 127]))
+        K = int(rng.integers(1, 12)) * 128 + int(rng.choice([0, 0, 8, 40, 120]))
+        N = int(rng.choice([1, 8, 16, 24, 32, 64]))
+        sp = float(rng.choice([0.0, 0.2, 0.4, 0.5, 0.5, 0.6, 0.7, 0.9, 0.99]))
+        kind = str(rng.choice(["magnitude", "bernoulli", "row_scaled", "wanda"]))
+        case = wl.Case(0, "soak", M, K, N, 500 + it, sp, kind)
+        W, X = case.make_W(), case.make_X()
+        if it % 3 == 0:
+            rows = rng.choice([0.0, 0.3, 1.0], size=(M + 31) // 32).repeat(32)[:M]
+            W = np.where(rng.random((M, K)) < rows[:, None], W, np.float16(0))
+        tag = f"case {it}: {M}x{K} N={N} sparsity {sp} {kind}"
+        ref = tl3.encode(W)
+        buf = torch.zeros((M, K + int(rng.choice([0, 8, 24]))), dtype=torch.float16, device="cuda")
+        buf[:, :K] = torch.from_numpy(W)
+        m = tl3.Matrix.encode_on_device(buf[:, :K])
+        for name in tl3.CANONICAL + tl3.COMPACT:
+            assert np.array_equal(m.canonical(name), ref.canonical(name)), (tag, name)
+        blob = m.upload_packed_on_device()
+        torch.cuda.synchronize()
+        assert np.array_equal(blob.cpu().numpy(), ref.pack()), tag
+        assert m.stats() == ref.stats(), tag
+        Xd = device_X(X)
+        Y = m.spmm(Xd).cpu().numpy()
+        check(oracle_mod, W, X, Y, with_oracle_spmm=False)
+        Yt = m.spmm_nt(Xd.t().contiguous()).cpu().numpy()
+        assert np.array_equal(Y.view(np.uint16), Yt.T.view(np.uint16)), tag
+        bias = (rng.standard_normal(M) * 0.1).astype(np.float16)
+        Yb = m.spmm(Xd, bias=torch.from_numpy(bias).cuda(), activation="relu").cpu().numpy().astype(np.float64)
+        Yref, bound = oracle_mod.dense_fp64(W, X)
+        want = np.maximum(Yref + bias.astype(np.float64)[:, None], 0.0)
+        assert np.all(np.abs(Yb - want) <= oracle_mod.tolerance(bound + np.abs(bias.astype(np.float64))[:, None])), tag
+        m.close()
+        ref.close()
