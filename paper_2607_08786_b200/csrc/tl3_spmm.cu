@@ -703,9 +703,13 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       // 16-byte stores when the columns fill them (N = 8 runs in the 16-column kernel)
       const bool vec_ok = !XT && (NPAD == 16 ? (a.N & 7) == 0 : a.N == NPAD) && (a.ldy & 7) == 0 && (reinterpret_cast<uintptr_t>(a.Y) & 15) == 0;
       const bool plain = a.bias == nullptr && a.act == TL3_ACT_NONE;
-      auto fin = [&](uint32_t bits) { const float f = __uint_as_float(bits); return plain ? f : finish(f, bias_v, a.act); };
-      auto store_y = [&](const uint32_t* v, int c0) {           // (bias, activation,) fp32 -> fp16 (round to nearest even) -> Y
+      auto fin = [](uint32_t bits) { return __uint_as_float(bits); };
+      auto store_y = [&](uint32_t* v, int c0) {                 // (bias, activation,) fp32 -> fp16 (round to nearest even) -> Y
         if (row >= a.M) return;
+        if (!plain) {                                             // one test per call, not one per element
+#pragma unroll
+          for (int c = 0; c < CH; ++c) v[c] = __float_as_uint(finish(__uint_as_float(v[c]), bias_v, a.act));
+        }
         if (vec_ok) {
 #pragma unroll
           for (int c = 0; c < CH; c += 8) {
@@ -786,12 +790,14 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
             }
           }
           __syncwarp();
+          if (et == 0) { TL3_GT(20) }
           if (staged && et == 0) mbar_arrive(bar_tail);           // the phase ends when every requested slot has landed
         }
         bool fetched = named_bar_all(1 + kGroups, 128, ok);
         if (staged) {
           if (fetched) {
             fetched = mbar_wait(bar_tail, 0, wctx, kStEpilogueTail);
+            if (et == 0) { TL3_GT(21) }
           } else if (et == 0) {                                   // giving up: still no exit with copies in flight
             for (uint32_t it = 0; it < (1u << 16) && !mbar_try_wait(bar_tail, 0); ++it) {}
           }
@@ -803,13 +809,20 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
             uint32_t v[CH];
             TmemLd<CH>::ld(acc_tmem + c0, v);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            for (int k = 0; k < n_others; ++k) {                  // own part first (lowest CTA), then ascending
-              if (staged) {
-                const uint32_t p = smem_base + (static_cast<uint32_t>(k) * NPAD * 128u + static_cast<uint32_t>(et)) * 4u;
+            // own part first (lowest CTA), then the others in ascending order.  Two loops: in one
+            // loop the slot arithmetic of the unstaged case (a 64-bit division per contributor)
+            // was computed on the staged path too, 0.25 us on a reducer's way out.
+            if (staged) {
+              uint32_t p = smem_base + static_cast<uint32_t>(et) * 4u + static_cast<uint32_t>(c0) * 512u;
+              for (int k = 0; k < n_others; ++k, p += NPAD * 512u) {
+                uint32_t w[CH];
 #pragma unroll
-                for (int c = 0; c < CH; ++c)
-                  v[c] = __float_as_uint(__uint_as_float(v[c]) + __uint_as_float(lds_u32(p + static_cast<uint32_t>(c0 + c) * 512u)));
-              } else {
+                for (int c = 0; c < CH; ++c) w[c] = lds_u32(p + static_cast<uint32_t>(c) * 512u);
+#pragma unroll
+                for (int c = 0; c < CH; ++c) v[c] = __float_as_uint(__uint_as_float(v[c]) + __uint_as_float(w[c]));
+              }
+            } else {
+              for (int k = 0; k < n_others; ++k) {
                 const int c_id = c_first + 1 + k;
                 const int sl = 2 * c_id + (range_begin(c_id, T, G) < row_tile_begin ? 1 : 0);
                 const float* p = a.partials + static_cast<size_t>(sl) * NPAD * 128 + et;
@@ -844,6 +857,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
         __threadfence();                                          // the partial sums, before the flag
         named_bar_sync(1 + kGroups, 128);
         if (et == 0) asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(a.flags + slot), "r"(1u) : "memory");
+        if (et == 0 && seg_end == t_end) { TL3_GT(22) }
       }
       ++seg;
       t = seg_end;
