@@ -60,6 +60,7 @@ constexpr int kClearWarp0 = 2;            // warps 2 and 3 clear the W_r buffers
 constexpr int kDecodeWarp0 = 4;           // warps 4-7: decode group 0, 8-11: group 1, ...
 constexpr int kEpilogueWarp0 = kDecodeWarp0 + 4 * kGroups;
 constexpr int kThreads = (kEpilogueWarp0 + 4) * 32;
+constexpr int kSetupBarrier = 2 + kGroups;   // named barriers: 0 = whole CTA, 1 + kGroups = epilogue warps, 2 + kGroups = set-up
 constexpr int kMaxStages = 8;
 constexpr uint32_t kWrBytes = 16384;
 constexpr int kMaxWrBuffers = 5;          // W_r ring: tile i uses buffer i % num_wr (4 or 5, see the launcher)
@@ -292,9 +293,11 @@ template <> struct TmemLd<64> {
   }
 };
 
-// CTA c of G owns tiles [c*T/G, (c+1)*T/G); the CTA that owns tile t:
-__device__ __forceinline__ long long range_begin(long long c, long long T, long long G) { return c * T / G; }
-__device__ __forceinline__ int owner_of(long long t, long long T, long long G) { return static_cast<int>(((t + 1) * G - 1) / T); }
+// CTA c of G owns tiles [c*T/G, (c+1)*T/G); the CTA that owns tile t.  In 32 bits: the launcher
+// refuses matrices with (G + 1) * T >= 2^32 (hundreds of gigabytes), and a 64-bit division costs a
+// CTA 0.15 us each at its cold start, where there are three of them.
+__device__ __forceinline__ uint32_t range_begin(uint32_t c, uint32_t T, uint32_t G) { return c * T / G; }
+__device__ __forceinline__ int owner_of(uint32_t t, uint32_t T, uint32_t G) { return static_cast<int>(((t + 1u) * G - 1u) / T); }
 
 // ---------------------------------------------------------------------------------------------
 // The kernel
@@ -399,8 +402,8 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) { TL3_GT(0) }
   if (tid == kEpilogueWarp0 * 32) { TL3_GT(1) TL3_GV(14, global_timer()) }
-  const long long T = a.total_tiles, G = gridDim.x;
-  const long long t_begin = range_begin(blockIdx.x, T, G), t_end = range_begin(blockIdx.x + 1, T, G);
+  const uint32_t T = static_cast<uint32_t>(a.total_tiles), G = gridDim.x;
+  const uint32_t t_begin = range_begin(blockIdx.x, T, G), t_end = range_begin(blockIdx.x + 1, T, G);
   const int n_tiles = static_cast<int>(t_end - t_begin);
   const int kt_begin = static_cast<int>(t_begin % a.tiles_k);
   // Decode groups in use: a group may wait for its next tile only once the stage's previous
@@ -409,29 +412,28 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   const int AG = S < kGroups ? S : kGroups;
   const uint32_t smem_base = smem_u32(smem);
 
-  if (tid == 0) {
-    for (int s = 0; s < kMaxStages; ++s) {
-      mbar_init(bar_full + 8 * s, 1);
-      mbar_init(bar_mma + 8 * s, 1);
-      mbar_init(bar_dec + 8 * s, 128);
-      mbar_init(bar_xfull + 8 * s, 1);
-    }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(bar_accfull + 8 * b, 1);
-      mbar_init(bar_accempty + 8 * b, 128);
-    }
-    for (int w = 0; w < kMaxWrBuffers; ++w) { mbar_init(bar_wrready + 8 * w, 64); mbar_init(bar_wrfree + 8 * w, 1); }
-    mbar_init(bar_tail, 1);
-    *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    TL3_GT(16)
-  }
-  // the producer's first directory entries and the X tensor map: start the (cold) global fetches
-  // before the set-up barrier
+  // Set-up.  The producer warp starts the (cold) global fetches of its first directory entries and
+  // of the X tensor map, initialises the barriers -- lane l words l and l + 32 of the block, two
+  // instructions instead of 57 in a row -- and goes on to request its first blocks without waiting
+  // for the tensor-memory allocation, which it does not use: it only arrives at the set-up barrier,
+  // the other warps wait there for it and for the allocating warp.
   uint4 dir_first = make_uint4(0, 0, 0, 0);
+  if (tid == 0) { TL3_GV(29, n_tiles + kt_begin) TL3_GT(28) }
   if (warp == kProducerWarp) {
     if (lane < n_tiles) dir_first = __ldg(reinterpret_cast<const uint4*>(a.dir + t_begin + lane));
     if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
+    if (lane == 0) { TL3_GT(30) }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int i = lane + 32 * h;                                // word of the barrier block (layout above)
+      const uint32_t count = i < 16 ? 1u : i < 24 ? 128u : i < 26 ? 1u : i < 28 ? 128u : i == 36 ? 1u
+                           : (i >= 44 && i < 44 + kMaxWrBuffers) ? 64u : (i >= 49 && i < 49 + kMaxWrBuffers) ? 1u : i >= 56 ? 1u : 0u;
+      if (count) mbar_init(smem_u32(bars + i), count);
+    }
+    if (lane == 0) *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) { TL3_GT(16) }
   }
   if (warp == kAllocWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
@@ -439,10 +441,11 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     if (lane == 0) { TL3_GT(19) }
   }
   tc_fence_before();
-  __syncthreads();
+  if (warp == kProducerWarp) asm volatile("bar.arrive %0, %1;" ::"r"(kSetupBarrier), "r"(kThreads) : "memory");
+  else named_bar_sync(kSetupBarrier, kThreads);
   tc_fence_after();
   if (tid == 0) { TL3_GT(17) }
-  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_base = warp == kProducerWarp ? 0u : *tmem_slot;   // (written by the allocating warp before it arrives)
   const WaitCtx wctx{abort_flag, a.status};
   pdl_launch_dependents();
 
@@ -466,17 +469,15 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
       }
       const int cnt = n_tiles - base < 32 ? n_tiles - base : 32;
       if (base == 0) {
-        for (int j = 0; j < pre; ++j) {                          // S <= 8 < 32: all in this batch
-          const uint32_t off16 = __shfl_sync(0xFFFFFFFFu, mine.x, j), bytes = __shfl_sync(0xFFFFFFFFu, mine.y, j);
-          if (lane == 0 && j == 0 && off16 != 0xFFFFFFFFu) { TL3_GT(18) }
-          const uint8_t* src = a.blob + static_cast<size_t>(off16) * 16;
-          const uint32_t st = smem_base + static_cast<uint32_t>(j) * a.stage_stride, full = bar_full + 8 * j;
-          if (elect_one()) {
-            mbar_arrive_expect_tx(full, split_x ? bytes : bytes + kXBytes);
-            bulk_copy_g2s(st, src, bytes, full);
-          }
-          __syncwarp();
+        // S <= 8 < 32: all in this batch, and lane j holds the entry of tile j -- the lanes request
+        // their blocks side by side (one after the other took 0.09 us per request)
+        if (lane == 0 && mine.x != 0xFFFFFFFFu) { TL3_GT(18) }
+        if (lane < pre) {
+          const uint32_t full = bar_full + 8 * lane;
+          mbar_arrive_expect_tx(full, split_x ? mine.y : mine.y + kXBytes);
+          bulk_copy_g2s(smem_base + static_cast<uint32_t>(lane) * a.stage_stride, a.blob + static_cast<size_t>(mine.x) * 16, mine.y, full);
         }
+        __syncwarp();
         if (lane == 0) { TL3_GT(2) }
         pdl_wait();
         if (lane == 0) { TL3_GT(3) }
@@ -678,12 +679,12 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
     const int et = tid - kEpilogueWarp0 * 32;                    // 0..127 = row of the tile = tensor-memory lane
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     int seg = 0;
-    long long t = t_begin;
+    uint32_t t = t_begin;
     pdl_wait();   // Y, the partial sums and their flags may still be in use by the previous kernel
     while (t < t_end) {
       const int mt = static_cast<int>(t / a.tiles_k);
-      const long long row_tile_begin = static_cast<long long>(mt) * a.tiles_k, row_tile_end = row_tile_begin + a.tiles_k;
-      const long long seg_end = row_tile_end < t_end ? row_tile_end : t_end;
+      const uint32_t row_tile_begin = static_cast<uint32_t>(mt) * static_cast<uint32_t>(a.tiles_k), row_tile_end = row_tile_begin + static_cast<uint32_t>(a.tiles_k);
+      const uint32_t seg_end = row_tile_end < t_end ? row_tile_end : t_end;
       const bool complete = (t == row_tile_begin) && (seg_end == row_tile_end);
       const int b = seg & 1;
       const int c_first = owner_of(row_tile_begin, T, G), c_last = owner_of(row_tile_end - 1, T, G);
@@ -1091,6 +1092,7 @@ static int spmm_block(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, 
 
   const long long total = m->n_tiles;
   const int grid = static_cast<int>(total < di.sm_count ? total : di.sm_count);
+  if (static_cast<unsigned long long>(total) * static_cast<unsigned long long>(grid + 1) >= (1ull << 32)) return TL3_ERR_UNSUPPORTED;   // the kernel splits the tiles in 32-bit arithmetic
   const WorkspaceLayout wl = workspace_layout(m, n_pad, di.sm_count);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   KernelArgs args;
