@@ -418,7 +418,7 @@ tl3_spmm_kernel(const __grid_constant__ CUtensorMap x_map, const KernelArgs a) {
   // for the tensor-memory allocation, which it does not use: it only arrives at the set-up barrier,
   // the other warps wait there for it and for the allocating warp.
   uint4 dir_first = make_uint4(0, 0, 0, 0);
-  if (tid == 0) { TL3_GV(29, n_tiles + kt_begin) TL3_GT(28) }
+  if (tid == 0) { TL3_GT(28) }                                   // (ranges known)
   if (warp == kProducerWarp) {
     if (lane < n_tiles) dir_first = __ldg(reinterpret_cast<const uint4*>(a.dir + t_begin + lane));
     if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
