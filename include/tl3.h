@@ -191,7 +191,8 @@ int tl3_workspace_init(void* workspace, size_t bytes, void* stream);
  * kernels hold SMs rests on the GPU dispatching the blocks of a grid in index order.
  * Threads: calls that take a const handle may share it; tl3_upload() and tl3_free() may not run
  * beside another call on the same handle.
- * Errors: NOT_UPLOADED, INVALID_ARG, UNSUPPORTED (N out of range, device is not sm_100), CUDA. */
+ * Errors: NOT_UPLOADED, INVALID_ARG, UNSUPPORTED (N out of range, device is not sm_100, or a matrix of
+ * 2^32 / (SMs + 1) tiles or more -- 28.8 million on B200, hundreds of gigabytes), CUDA. */
 #define TL3_MAX_N 4096
 int tl3_spmm(const tl3_matrix* m, const void* X, int64_t ldx, void* Y, int64_t ldy, int N,
              void* workspace, void* stream);
