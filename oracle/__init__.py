@@ -7,6 +7,7 @@ from .oracle import (  # noqa: F401
     Container,
     build,
     compact_nbytes,
+    compact_nbytes_all,
     decode,
     dense_fp64,
     encode,
@@ -17,4 +18,6 @@ from .oracle import (  # noqa: F401
     spmm,
     threads,
     tolerance,
+    values_compact,
+    values_expand,
 )

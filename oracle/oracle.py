@@ -260,6 +260,80 @@ def residual_expand(c: Container, res_dir, res_list, res_mask) -> np.ndarray:
     return out
 
 
+# --- Empty value slots above 50 % sparsity (the paper's Sec. 6: "most regions require zero padding").
+# The paper stores every slot of the Sparse-TC value array; a slot that neither keeps a weight nor
+# had one parked in it holds zero.  Compact form (a reading, like the Residual's): per tile either
+# the tile's tile_m * H values as they are, or a bitmap of the occupied slots (bit pos % 8 of byte
+# pos // 8, pos = row * H + slot, the coordinate of the PDD streams) followed by the occupied
+# slots' values in ascending position order; the bitmap is taken iff it is strictly smaller, i.e.
+# iff its bytes are fewer than two per empty slot.  "Occupied" = value bits & 0x7FFF != 0.
+def values_compact(c: Container):
+    """(val_dir, val_pack, val_mask) of a container's Sparse-TC value array.
+
+    val_dir  u32[tiles][2]  {mode, off}: mode 0 = all tile_m * H values of the tile, starting at
+                            val_pack[off]; mode 1 = only the occupied slots' values, starting at
+                            val_pack[off], and the tile's bitmap at val_mask[index * B] where index
+                            counts the bitmap-mode tiles before this one
+    val_pack u16[]          values, tile after tile, row-major inside a tile
+    val_mask u8[]           B = ceil(tile_m * H / 8) bytes per bitmap-mode tile"""
+    H = c.tile_k // 2
+    S = c.tile_m * H
+    B = (S + 7) // 8
+    tiles_m, tiles_k = c.M_pad // c.tile_m, c.K_pad // c.tile_k
+    vals = np.asarray(c.tc_vals, dtype=np.uint16).reshape(c.M_pad, c.K_pad // 2)
+    val_dir = np.zeros((tiles_m * tiles_k, 2), dtype=np.uint32)
+    packs, masks = [], []
+    n_pack = 0
+    for tm in range(tiles_m):
+        for tk in range(tiles_k):
+            t = tm * tiles_k + tk
+            tile = vals[tm * c.tile_m:(tm + 1) * c.tile_m, tk * H:(tk + 1) * H].reshape(-1)
+            occupied = (tile & 0x7FFF) != 0
+            empties = S - int(occupied.sum())
+            if B < 2 * empties:
+                masks.append(np.packbits(occupied.astype(np.uint8), bitorder="little"))
+                packs.append(tile[occupied])
+                val_dir[t] = (1, n_pack)
+                n_pack += int(occupied.sum())
+            else:
+                packs.append(tile.copy())
+                val_dir[t] = (0, n_pack)
+                n_pack += S
+    val_pack = np.concatenate(packs) if packs else np.zeros(0, dtype=np.uint16)
+    val_mask = np.concatenate(masks) if masks else np.zeros(0, dtype=np.uint8)
+    return val_dir, val_pack.astype(np.uint16), val_mask.astype(np.uint8)
+
+
+def values_expand(c: Container, val_dir, val_pack, val_mask) -> np.ndarray:
+    """The inverse: the full value array tc_vals (u16, M_pad * K_pad / 2) from the compact form.
+    An empty slot comes back as +0.0, which is what the encoder writes there."""
+    H = c.tile_k // 2
+    S = c.tile_m * H
+    B = (S + 7) // 8
+    tiles_m, tiles_k = c.M_pad // c.tile_m, c.K_pad // c.tile_k
+    out = np.zeros((c.M_pad, c.K_pad // 2), dtype=np.uint16)
+    n_mask = 0
+    for tm in range(tiles_m):
+        for tk in range(tiles_k):
+            t = tm * tiles_k + tk
+            mode, at = int(val_dir[t, 0]), int(val_dir[t, 1])
+            if mode == 1:
+                bits = np.unpackbits(np.asarray(val_mask[n_mask * B:(n_mask + 1) * B], dtype=np.uint8), bitorder="little")[:S].astype(bool)
+                n_mask += 1
+                tile = np.zeros(S, dtype=np.uint16)
+                tile[bits] = val_pack[at:at + int(bits.sum())]
+            else:
+                tile = np.asarray(val_pack[at:at + S], dtype=np.uint16)
+            out[tm * c.tile_m:(tm + 1) * c.tile_m, tk * H:(tk + 1) * H] = tile.reshape(c.tile_m, H)
+    return out.reshape(-1)
+
+
+def compact_nbytes_all(c: Container) -> int:
+    """Size of the container with the Residual layer and the value array in their compact forms."""
+    val_dir, val_pack, val_mask = values_compact(c)
+    return compact_nbytes(c) - np.asarray(c.tc_vals, dtype=np.uint16).nbytes + val_dir.nbytes + val_pack.nbytes + val_mask.nbytes
+
+
 def compact_nbytes(c: Container) -> int:
     """Size of the container with the Residual layer in its compact form."""
     res_dir, res_list, res_mask = residual_compact(c)
