@@ -591,7 +591,11 @@ def _point(tl3, dev, peak, case, verify_rows=0):
     row = _row(wt, case.N, us, dus, peak)
     st = wt.stats
     row.update({"name": case.name, "sf_share": round(st["n_sf"] / st["nnz"], 4), "res_share": round(st["n_res"] / st["nnz"], 4),
-                "host_encode_s": round(wt.encode_s, 2), "device_pack_upload_s": round(wt.upload_s, 2)})
+                "host_encode_s": round(wt.encode_s, 2), "device_pack_upload_s": round(wt.upload_s, 2),
+                # the container on disk: as the paper stores it, and with the Residual layer and the
+                # value array in their compact forms (the kernel streams the device image above)
+                "container_over_dense": round(st["canonical_bytes"] / (2 * case.M * case.K), 4),
+                "container_compact_over_dense": round(st["canonical_bytes_compact_all"] / (2 * case.M * case.K), 4)})
     if verify_rows:
         rows = np.random.default_rng(case.seed).choice(case.M, size=verify_rows, replace=False)
         Wr = wt.W[rows].astype(np.float64)

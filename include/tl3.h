@@ -53,6 +53,7 @@ typedef struct {
   int64_t dev_n_res;          /* elements that travel as Residual entries                           */
   int64_t dev_n_dummy;        /* delta bytes that move nothing: dummy points and chain padding      */
   int64_t dev_pdd_bytes;      /* delta bytes in all                                                 */
+  int64_t canonical_bytes_compact_all;  /* canonical_bytes_compact with the value array in its compact form too */
 } tl3_stats_t;
 
 enum {
@@ -84,8 +85,17 @@ enum {
   TL3_RES_DIR = 9,     /* u32 [tiles][2]        {mode, off}: 0 = list, off indexes TL3_RES_LIST;        */
                        /*                       1 = bitmap, off = byte offset into TL3_RES_MASK         */
   TL3_RES_LIST = 10,   /* u16 []                positions of the list-mode tiles                         */
-  TL3_RES_MASK = 11    /* u8  []                ceil(tile_m*tile_k/16) bytes per bitmap-mode tile, bit   */
+  TL3_RES_MASK = 11,   /* u8  []                ceil(tile_m*tile_k/16) bytes per bitmap-mode tile, bit   */
                        /*                       rho % 8 of byte rho / 8                                  */
+  /* Compact form of the Sparse-TC value array, derived from TL3_TC_VALS.  The paper stores every
+   * slot (Sec. 3.2) and names the slots that stay empty above 50 % sparsity as a limitation
+   * (Sec. 6).  Per tile whichever is smaller: all tile_m * tile_k / 2 values, or a bitmap of the
+   * occupied slots (value bits & 0x7FFF != 0; bit pos % 8 of byte pos / 8, pos = row * tile_k / 2 +
+   * slot) plus the occupied slots' values in ascending position order. */
+  TL3_VAL_DIR = 12,    /* u32 [tiles][2]        {mode, off}: off indexes TL3_VAL_PACK; 0 = all values,  */
+                       /*                       1 = occupied slots only, bitmaps in tile order           */
+  TL3_VAL_PACK = 13,   /* u16 []                values, tile after tile                                  */
+  TL3_VAL_MASK = 14    /* u8  []                ceil(tile_m*tile_k/16) bytes per bitmap-mode tile        */
 };
 
 /* ---- format: host side (Sec. 3.2) ------------------------------------------------------ */

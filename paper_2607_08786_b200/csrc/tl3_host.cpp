@@ -393,10 +393,55 @@ static void ensure_compact(const tl3_matrix* m) {
   m->compact_ready.store(true, std::memory_order_release);
 }
 
+// Compact form of the value array (Sec. 3.2 stores every slot; Sec. 6 names the empty ones above
+// 50 % sparsity): per tile all values, or a bitmap of the occupied slots and their values,
+// whichever is smaller.
+static void ensure_val_compact(const tl3_matrix* m) {
+  if (m->val_compact_ready.load(std::memory_order_acquire)) return;
+  std::lock_guard<std::mutex> lock(m->layout_mu);
+  if (m->val_compact_ready.load(std::memory_order_relaxed)) return;
+  const int64_t H = m->p.tile_k / 2, slots = static_cast<int64_t>(m->p.tile_m) * H, half_ld = m->K_pad / 2;
+  const size_t mask_bytes = (static_cast<size_t>(slots) + 7) / 8;
+  const int64_t tiles_k = m->K_pad / m->p.tile_k;
+  m->val_dir.assign(static_cast<size_t>(m->n_tiles) * 2, 0);
+  m->val_pack.clear();
+  m->val_mask.clear();
+  for (int64_t t = 0; t < m->n_tiles; ++t) {
+    const int64_t tm = t / tiles_k, tk = t % tiles_k;
+    const uint16_t* base = m->tc_vals.data() + tm * m->p.tile_m * half_ld + tk * H;
+    int64_t occupied = 0;
+    for (int64_t r = 0; r < m->p.tile_m; ++r)
+      for (int64_t h = 0; h < H; ++h) occupied += (base[r * half_ld + h] & 0x7FFFu) != 0;
+    const bool bitmap = mask_bytes < 2u * static_cast<size_t>(slots - occupied);
+    m->val_dir[2 * t] = bitmap ? 1u : 0u;
+    m->val_dir[2 * t + 1] = static_cast<uint32_t>(m->val_pack.size());
+    uint8_t* bits = nullptr;
+    if (bitmap) {
+      m->val_mask.resize(m->val_mask.size() + mask_bytes, 0);
+      bits = m->val_mask.data() + m->val_mask.size() - mask_bytes;
+    }
+    for (int64_t r = 0; r < m->p.tile_m; ++r)
+      for (int64_t h = 0; h < H; ++h) {
+        const uint16_t v = base[r * half_ld + h];
+        if (!bitmap) { m->val_pack.push_back(v); continue; }
+        if ((v & 0x7FFFu) != 0) {
+          const int64_t pos = r * H + h;
+          bits[pos >> 3] |= static_cast<uint8_t>(1u << (pos & 7));
+          m->val_pack.push_back(v);
+        }
+      }
+  }
+  m->val_compact_ready.store(true, std::memory_order_release);
+}
+
 int tl3_canonical(const tl3_matrix* m, int which, const void** ptr, size_t* bytes) {
   if (!m || !ptr || !bytes) return TL3_ERR_INVALID_ARG;
   if (which >= TL3_RES_DIR && which <= TL3_RES_MASK) ensure_compact(m);
+  if (which >= TL3_VAL_DIR && which <= TL3_VAL_MASK) ensure_val_compact(m);
   switch (which) {
+    case TL3_VAL_DIR:    *ptr = m->val_dir.data();    *bytes = m->val_dir.size() * 4; break;
+    case TL3_VAL_PACK:   *ptr = m->val_pack.data();   *bytes = m->val_pack.size() * 2; break;
+    case TL3_VAL_MASK:   *ptr = m->val_mask.data();   *bytes = m->val_mask.size(); break;
     case TL3_RES_DIR:    *ptr = m->res_dir.data();    *bytes = m->res_dir.size() * 4; break;
     case TL3_RES_LIST:   *ptr = m->res_list.data();   *bytes = m->res_list.size() * 2; break;
     case TL3_RES_MASK:   *ptr = m->res_mask.data();   *bytes = m->res_mask.size(); break;
@@ -432,6 +477,9 @@ int tl3_stats(const tl3_matrix* m, tl3_stats_t* out) {
                                  static_cast<int64_t>(m->res_dir.size() * 4 + m->res_list.size() * 2 + m->res_mask.size());
   out->dev_n_sf = m->dev_n_sf; out->dev_n_res = m->dev_n_res; out->dev_n_dummy = m->dev_n_dummy;
   out->dev_pdd_bytes = m->dev_pdd_bytes;
+  ensure_val_compact(m);
+  out->canonical_bytes_compact_all = out->canonical_bytes_compact - static_cast<int64_t>(m->tc_vals.size() * 2) +
+                                     static_cast<int64_t>(m->val_dir.size() * 4 + m->val_pack.size() * 2 + m->val_mask.size());
   return TL3_OK;
 }
 

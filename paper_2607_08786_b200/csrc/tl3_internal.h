@@ -47,6 +47,10 @@ struct tl3_matrix {
   mutable std::vector<uint32_t> res_dir;
   mutable std::vector<uint16_t> res_list;
   mutable std::vector<uint8_t> res_mask;
+  mutable std::atomic<bool> val_compact_ready{false};      // compact form of the value array (tl3_canonical 12-14)
+  mutable std::vector<uint32_t> val_dir;
+  mutable std::vector<uint16_t> val_pack;
+  mutable std::vector<uint8_t> val_mask;
 
   // last launch geometry (reporting only)
   mutable std::atomic<int> last_ctas{0}, last_stages{0}, last_smem{0};

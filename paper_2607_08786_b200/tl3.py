@@ -23,8 +23,10 @@ CANONICAL = ("tc_vals", "tc_meta", "chain_tau0", "chain_rho0", "chain_len", "pdd
              "res_rho", "res_val")
 # the compact form of the Residual layer, derived from res_rho (numbered after the nine above)
 COMPACT = ("res_dir", "res_list", "res_mask")
+# the compact form of the Sparse-TC value array, derived from tc_vals (numbered after those)
+COMPACT_VALUES = ("val_dir", "val_pack", "val_mask")
 _CANONICAL_DTYPES = (np.uint16, np.uint8, np.uint16, np.uint16, np.uint8, np.uint8, np.uint32,
-                     np.uint16, np.uint16, np.uint32, np.uint16, np.uint8)
+                     np.uint16, np.uint16, np.uint32, np.uint16, np.uint8, np.uint32, np.uint16, np.uint8)
 
 # every symbol include/tl3.h declares
 SYMBOLS = ("tl3_encode", "tl3_encode_device", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_deserialize",
@@ -61,7 +63,7 @@ class Stats(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in
                 ("M", "K", "M_pad", "K_pad", "n_tiles", "nnz", "n_tc", "n_sf", "n_res", "n_dummy",
                  "n_slots_unused", "canonical_bytes", "device_bytes", "canonical_bytes_compact",
-                 "dev_n_sf", "dev_n_res", "dev_n_dummy", "dev_pdd_bytes")]
+                 "dev_n_sf", "dev_n_res", "dev_n_dummy", "dev_pdd_bytes", "canonical_bytes_compact_all")]
 
     def as_dict(self) -> dict:
         return {n: int(getattr(self, n)) for n, _ in self._fields_}
@@ -212,7 +214,7 @@ class Matrix:
         return W
 
     def canonical(self, which) -> np.ndarray:
-        idx = (CANONICAL + COMPACT).index(which) if isinstance(which, str) else int(which)
+        idx = (CANONICAL + COMPACT + COMPACT_VALUES).index(which) if isinstance(which, str) else int(which)
         p, n = ctypes.c_void_p(), ctypes.c_size_t()
         _check(lib().tl3_canonical(self._h, idx, ctypes.byref(p), ctypes.byref(n)), "tl3_canonical")
         if n.value == 0:

@@ -192,6 +192,26 @@ def test_compact_residual_matches_the_oracle(tl3, oracle_mod, sparsity):
     assert st["dev_n_res"] >= st["n_res"] and 0 <= st["dev_n_dummy"] <= st["dev_pdd_bytes"]
 
 
+@pytest.mark.parametrize("sparsity,tiles", [(0.5, (128, 128)), (0.6, (128, 128)), (0.7, (128, 128)), (0.7, (4, 32))])
+def test_compact_values_match_the_oracle(tl3, oracle_mod, sparsity, tiles):
+    """The library's compact form of the Sparse-TC value array (all values, or a bitmap of the
+    occupied slots and their values, per tile) byte for byte against the oracle's, on a ragged
+    shape, and the size tl3_stats reports against the oracle's."""
+    W = wl.Case(0, "cv", 300, 520, 8, 21, sparsity, "magnitude").make_W()
+    m = tl3.encode(W, tile_m=tiles[0], tile_k=tiles[1])
+    cont = oracle_mod.encode(W, *tiles)
+    val_dir, val_pack, val_mask = oracle_mod.values_compact(cont)
+    assert np.array_equal(m.canonical("val_dir").reshape(-1, 2), val_dir)
+    assert np.array_equal(m.canonical("val_pack"), val_pack)
+    assert np.array_equal(m.canonical("val_mask"), val_mask)
+    assert m.stats()["canonical_bytes_compact_all"] == oracle_mod.compact_nbytes_all(cont)
+    # above 50 % every tile takes the bitmap; at 50 % an interior tile does not (the ragged edge's
+    # padded tiles, mostly empty, do)
+    assert (val_dir[:, 0] == 1).all() if sparsity > 0.5 else val_dir[0, 0] == 0
+    assert np.array_equal(oracle_mod.values_expand(cont, m.canonical("val_dir").reshape(-1, 2), m.canonical("val_pack"),
+                                                   m.canonical("val_mask")), m.canonical("tc_vals"))
+
+
 def test_launch_tuning_round_trip(tl3):
     L = tl3.lib()
     assert tl3.get_tuning() == {"decode_before_x": 4}
