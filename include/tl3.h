@@ -90,7 +90,7 @@ enum {
   /* Compact form of the Sparse-TC value array, derived from TL3_TC_VALS.  The paper stores every
    * slot (Sec. 3.2) and names the slots that stay empty above 50 % sparsity as a limitation
    * (Sec. 6).  Per tile whichever is smaller: all tile_m * tile_k / 2 values, or a bitmap of the
-   * occupied slots (value bits & 0x7FFF != 0; bit pos % 8 of byte pos / 8, pos = row * tile_k / 2 +
+   * occupied slots (value bits != 0; bit pos % 8 of byte pos / 8, pos = row * tile_k / 2 +
    * slot) plus the occupied slots' values in ascending position order. */
   TL3_VAL_DIR = 12,    /* u32 [tiles][2]        {mode, off}: off indexes TL3_VAL_PACK; 0 = all values,  */
                        /*                       1 = occupied slots only, bitmaps in tile order           */

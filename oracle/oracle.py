@@ -266,7 +266,9 @@ def residual_expand(c: Container, res_dir, res_list, res_mask) -> np.ndarray:
 # the tile's tile_m * H values as they are, or a bitmap of the occupied slots (bit pos % 8 of byte
 # pos // 8, pos = row * H + slot, the coordinate of the PDD streams) followed by the occupied
 # slots' values in ascending position order; the bitmap is taken iff it is strictly smaller, i.e.
-# iff its bytes are fewer than two per empty slot.  "Occupied" = value bits & 0x7FFF != 0.
+# iff its bytes are fewer than two per empty slot.  "Occupied" = any non-zero bit pattern (the
+# encoder writes +0.0 into an empty slot; a container that carries -0.0 there keeps it, so the
+# compact form is lossless for every container).
 def values_compact(c: Container):
     """(val_dir, val_pack, val_mask) of a container's Sparse-TC value array.
 
@@ -288,7 +290,7 @@ def values_compact(c: Container):
         for tk in range(tiles_k):
             t = tm * tiles_k + tk
             tile = vals[tm * c.tile_m:(tm + 1) * c.tile_m, tk * H:(tk + 1) * H].reshape(-1)
-            occupied = (tile & 0x7FFF) != 0
+            occupied = tile != 0
             empties = S - int(occupied.sum())
             if B < 2 * empties:
                 masks.append(np.packbits(occupied.astype(np.uint8), bitorder="little"))
@@ -305,8 +307,8 @@ def values_compact(c: Container):
 
 
 def values_expand(c: Container, val_dir, val_pack, val_mask) -> np.ndarray:
-    """The inverse: the full value array tc_vals (u16, M_pad * K_pad / 2) from the compact form.
-    An empty slot comes back as +0.0, which is what the encoder writes there."""
+    """The inverse: the full value array tc_vals (u16, M_pad * K_pad / 2) from the compact form
+    (an empty slot is the bit pattern 0)."""
     H = c.tile_k // 2
     S = c.tile_m * H
     B = (S + 7) // 8

@@ -411,7 +411,7 @@ static void ensure_val_compact(const tl3_matrix* m) {
     const uint16_t* base = m->tc_vals.data() + tm * m->p.tile_m * half_ld + tk * H;
     int64_t occupied = 0;
     for (int64_t r = 0; r < m->p.tile_m; ++r)
-      for (int64_t h = 0; h < H; ++h) occupied += (base[r * half_ld + h] & 0x7FFFu) != 0;
+      for (int64_t h = 0; h < H; ++h) occupied += base[r * half_ld + h] != 0;
     const bool bitmap = mask_bytes < 2u * static_cast<size_t>(slots - occupied);
     m->val_dir[2 * t] = bitmap ? 1u : 0u;
     m->val_dir[2 * t + 1] = static_cast<uint32_t>(m->val_pack.size());
@@ -424,7 +424,7 @@ static void ensure_val_compact(const tl3_matrix* m) {
       for (int64_t h = 0; h < H; ++h) {
         const uint16_t v = base[r * half_ld + h];
         if (!bitmap) { m->val_pack.push_back(v); continue; }
-        if ((v & 0x7FFFu) != 0) {
+        if (v != 0) {
           const int64_t pos = r * H + h;
           bits[pos >> 3] |= static_cast<uint8_t>(1u << (pos & 7));
           m->val_pack.push_back(v);

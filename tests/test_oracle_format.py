@@ -411,6 +411,11 @@ def test_compact_values_round_trip_and_size_rule(oracle_mod):
         c = _values_container(oracle_mod, M, K, tile_m, tile_k, vals)
         val_dir, val_pack, val_mask = oracle_mod.values_compact(c)
         assert np.array_equal(oracle_mod.values_expand(c, val_dir, val_pack, val_mask), vals.reshape(-1))
+        # a slot that holds -0.0 is a bit pattern to keep: the form is lossless for every container
+        v2 = vals.copy()
+        v2[0, 0] = 0x8000
+        c2 = _values_container(oracle_mod, M, K, tile_m, tile_k, v2)
+        assert np.array_equal(oracle_mod.values_expand(c2, *oracle_mod.values_compact(c2)), v2.reshape(-1))
         at_pack = at_mask = 0
         for t, at in enumerate(occ):
             bitmap = B < 2 * (S - len(at))
