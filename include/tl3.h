@@ -130,6 +130,14 @@ int tl3_stats(const tl3_matrix* m, tl3_stats_t* out);
  * tl3_serialize: buf == NULL writes the needed size to *bytes; otherwise *bytes is the capacity
  * on entry and the size written on return.  buf: host. */
 int tl3_serialize(const tl3_matrix* m, void* buf, size_t* bytes);
+/* The same container with the Residual positions and the value array in their compact forms
+ * (TL3_RES_DIR ... TL3_VAL_MASK): what to write to disk or send below 50 % and above 50 %
+ * sparsity (0.81 -> 0.75 x dense at 40 %, 0.61 -> 0.54 at 60 %, 0.59 -> 0.43 at 70 %; the same
+ * size as tl3_serialize plus two small directories at 50 %).  Same calling convention. */
+int tl3_serialize_compact(const tl3_matrix* m, void* buf, size_t* bytes);
+/* Reads either form (the header says which) into a new handle whose nine canonical arrays are
+ * those of the container that was written, bit for bit.  Errors: INVALID_ARG, BAD_CONTAINER
+ * (truncated, inconsistent or out-of-range contents; nothing is trusted), NO_MEMORY. */
 int tl3_deserialize(const void* buf, size_t bytes, tl3_matrix** out);
 
 void tl3_free(tl3_matrix* m);

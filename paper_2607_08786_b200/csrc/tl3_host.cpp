@@ -522,6 +522,100 @@ int tl3_serialize(const tl3_matrix* m, void* buf, size_t* bytes) {
   return TL3_OK;
 }
 
+// The compact form on disk: header (reserved = 1) and thirteen arrays.
+static const int kCompactOrder[13] = {TL3_VAL_DIR, TL3_VAL_PACK, TL3_VAL_MASK, TL3_TC_META, TL3_CHAIN_TAU0, TL3_CHAIN_RHO0, TL3_CHAIN_LEN,
+                                      TL3_PDD_BYTES, TL3_TILE_DIR, TL3_RES_DIR, TL3_RES_LIST, TL3_RES_MASK, TL3_RES_VAL};
+
+int tl3_serialize_compact(const tl3_matrix* m, void* buf, size_t* bytes) {
+  if (!m || !bytes) return TL3_ERR_INVALID_ARG;
+  size_t need = sizeof(FileHeader);
+  for (int w : kCompactOrder) {
+    const void* p; size_t n;
+    tl3_canonical(m, w, &p, &n);
+    need += sizeof(uint64_t) + n;
+  }
+  if (!buf) { *bytes = need; return TL3_OK; }
+  if (*bytes < need) { *bytes = need; return TL3_ERR_INVALID_ARG; }
+  uint8_t* o = static_cast<uint8_t*>(buf);
+  FileHeader h{kMagic, m->M, m->K, m->p.tile_m, m->p.tile_k, m->p.maxd, 1,
+               {m->nnz, m->n_tc, m->n_sf, m->n_res, m->n_dummy, m->n_slots_unused}};
+  std::memcpy(o, &h, sizeof(h));
+  o += sizeof(h);
+  for (int w : kCompactOrder) {
+    const void* p; size_t n;
+    tl3_canonical(m, w, &p, &n);
+    const uint64_t n64 = n;
+    std::memcpy(o, &n64, 8);
+    o += 8;
+    if (n) std::memcpy(o, p, n);
+    o += n;
+  }
+  *bytes = need;
+  return TL3_OK;
+}
+
+// Expands the compact arrays of a container that was just read; false if anything is out of range.
+static bool expand_compact(tl3_matrix& m, const std::vector<uint32_t>& val_dir, const std::vector<uint16_t>& val_pack,
+                           const std::vector<uint8_t>& val_mask, const std::vector<uint32_t>& res_dir,
+                           const std::vector<uint16_t>& res_list, const std::vector<uint8_t>& res_mask) {
+  const int64_t H = m.p.tile_k / 2, slots = static_cast<int64_t>(m.p.tile_m) * H, half_ld = m.K_pad / 2;
+  const size_t mask_bytes = (static_cast<size_t>(slots) + 7) / 8;
+  const int64_t tiles_k = m.K_pad / m.p.tile_k;
+  const size_t nt = static_cast<size_t>(m.n_tiles);
+  if (val_dir.size() != 2 * nt || res_dir.size() != 2 * nt || m.tile_dir.size() != 4 * nt) return false;
+  m.tc_vals.assign(static_cast<size_t>(m.M_pad) * static_cast<size_t>(half_ld), 0);
+  size_t n_mask = 0, expect_pack = 0;
+  for (size_t t = 0; t < nt; ++t) {
+    const uint32_t mode = val_dir[2 * t], off = val_dir[2 * t + 1];
+    if (mode > 1 || off != expect_pack) return false;               // tiles follow each other in val_pack
+    const int64_t tm = static_cast<int64_t>(t) / tiles_k, tk = static_cast<int64_t>(t) % tiles_k;
+    uint16_t* base = m.tc_vals.data() + tm * m.p.tile_m * half_ld + tk * H;
+    if (mode == 0) {
+      if (val_pack.size() - off < static_cast<size_t>(slots)) return false;
+      for (int64_t r = 0; r < m.p.tile_m; ++r) std::memcpy(base + r * half_ld, val_pack.data() + off + r * H, static_cast<size_t>(H) * 2);
+      expect_pack += static_cast<size_t>(slots);
+    } else {
+      if (val_mask.size() / mask_bytes <= n_mask) return false;
+      const uint8_t* bits = val_mask.data() + n_mask * mask_bytes;
+      ++n_mask;
+      size_t at = off;
+      for (int64_t pos = 0; pos < slots; ++pos) {
+        if (!((bits[pos >> 3] >> (pos & 7)) & 1u)) continue;
+        if (at >= val_pack.size() || val_pack[at] == 0) return false;  // an occupied slot holds a non-zero pattern
+        base[(pos / H) * half_ld + pos % H] = val_pack[at++];
+      }
+      for (int64_t pos = slots; pos < static_cast<int64_t>(mask_bytes) * 8; ++pos)
+        if ((bits[pos >> 3] >> (pos & 7)) & 1u) return false;          // bits beyond the tile
+      expect_pack = at;
+    }
+  }
+  if (expect_pack != val_pack.size() || n_mask * mask_bytes != val_mask.size()) return false;
+  m.res_rho.assign(m.res_val.size(), 0);
+  size_t expect_list = 0, expect_mask = 0;
+  for (size_t t = 0; t < nt; ++t) {
+    const uint32_t off = m.tile_dir[4 * t + 2], cnt = m.tile_dir[4 * t + 3];
+    const uint32_t mode = res_dir[2 * t], at = res_dir[2 * t + 1];
+    if (mode > 1 || static_cast<size_t>(off) + cnt > m.res_rho.size()) return false;
+    if (mode == 0) {
+      if (at != expect_list || res_list.size() - at < cnt) return false;
+      std::memcpy(m.res_rho.data() + off, res_list.data() + at, static_cast<size_t>(cnt) * 2);
+      expect_list += cnt;
+    } else {
+      if (at != expect_mask || res_mask.size() - at < mask_bytes) return false;
+      const uint8_t* bits = res_mask.data() + at;
+      uint32_t k = 0;
+      for (int64_t pos = 0; pos < static_cast<int64_t>(mask_bytes) * 8; ++pos) {
+        if (!((bits[pos >> 3] >> (pos & 7)) & 1u)) continue;
+        if (pos >= slots || k >= cnt) return false;
+        m.res_rho[off + k++] = static_cast<uint16_t>(pos);
+      }
+      if (k != cnt) return false;
+      expect_mask += mask_bytes;
+    }
+  }
+  return expect_list == res_list.size() && expect_mask == res_mask.size();
+}
+
 int tl3_deserialize(const void* buf, size_t bytes, tl3_matrix** out) {
   if (!buf || !out) return TL3_ERR_INVALID_ARG;
   if (bytes < sizeof(FileHeader)) return TL3_ERR_BAD_CONTAINER;
@@ -552,8 +646,17 @@ int tl3_deserialize(const void* buf, size_t bytes, tl3_matrix** out) {
   };
   bool ok = false;
   try {
-    ok = read(m->tc_vals) && read(m->tc_meta) && read(m->chain_tau0) && read(m->chain_rho0) &&
-         read(m->chain_len) && read(m->pdd_bytes) && read(m->tile_dir) && read(m->res_rho) && read(m->res_val);
+    if (h.reserved == 0) {
+      ok = read(m->tc_vals) && read(m->tc_meta) && read(m->chain_tau0) && read(m->chain_rho0) &&
+           read(m->chain_len) && read(m->pdd_bytes) && read(m->tile_dir) && read(m->res_rho) && read(m->res_val);
+    } else if (h.reserved == 1) {                                   // compact form (tl3_serialize_compact)
+      std::vector<uint32_t> val_dir, res_dir;
+      std::vector<uint16_t> val_pack, res_list;
+      std::vector<uint8_t> val_mask, res_mask;
+      ok = read(val_dir) && read(val_pack) && read(val_mask) && read(m->tc_meta) && read(m->chain_tau0) && read(m->chain_rho0) &&
+           read(m->chain_len) && read(m->pdd_bytes) && read(m->tile_dir) && read(res_dir) && read(res_list) && read(res_mask) &&
+           read(m->res_val) && expand_compact(*m, val_dir, val_pack, val_mask, res_dir, res_list, res_mask);
+    }
   } catch (const std::bad_alloc&) {
     delete m;
     return TL3_ERR_NO_MEMORY;

@@ -29,7 +29,7 @@ _CANONICAL_DTYPES = (np.uint16, np.uint8, np.uint16, np.uint16, np.uint8, np.uin
                      np.uint16, np.uint16, np.uint32, np.uint16, np.uint8, np.uint32, np.uint16, np.uint8)
 
 # every symbol include/tl3.h declares
-SYMBOLS = ("tl3_encode", "tl3_encode_device", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_deserialize",
+SYMBOLS = ("tl3_encode", "tl3_encode_device", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_serialize_compact", "tl3_deserialize",
            "tl3_free", "tl3_device_bytes", "tl3_pack", "tl3_upload", "tl3_bind", "tl3_plan_device", "tl3_upload_device", "tl3_workspace_bytes", "tl3_workspace_init",
            "tl3_spmm", "tl3_spmm_ex", "tl3_spmm_nt", "tl3_spmm_host", "tl3_spmm_host_async", "tl3_spmm_static_scratch", "tl3_static_scratch_status", "tl3_status", "tl3_status_word", "tl3_selftest_bounded_wait", "tl3_last_launch", "tl3_strerror",
            "tl3_last_cuda_error", "tl3_get_tuning", "tl3_set_tuning")
@@ -87,6 +87,7 @@ def lib() -> ctypes.CDLL:
         L.tl3_canonical.argtypes = [vp, ci, ctypes.POINTER(vp), ctypes.POINTER(sz)]
         L.tl3_stats.argtypes = [vp, ctypes.POINTER(Stats)]
         L.tl3_serialize.argtypes = [vp, vp, ctypes.POINTER(sz)]
+        L.tl3_serialize_compact.argtypes = [vp, vp, ctypes.POINTER(sz)]
         L.tl3_deserialize.argtypes = [vp, sz, ctypes.POINTER(vp)]
         L.tl3_free.argtypes = [vp]
         L.tl3_free.restype = None
@@ -222,11 +223,14 @@ class Matrix:
         buf = (ctypes.c_uint8 * n.value).from_address(p.value)
         return np.frombuffer(buf, dtype=_CANONICAL_DTYPES[idx]).copy()
 
-    def serialize(self) -> bytes:
+    def serialize(self, compact: bool = False) -> bytes:
+        """The container as bytes; ``compact=True`` writes the Residual positions and the value
+        array in their compact forms (``deserialize`` reads both)."""
+        fn = lib().tl3_serialize_compact if compact else lib().tl3_serialize
         n = ctypes.c_size_t()
-        _check(lib().tl3_serialize(self._h, None, ctypes.byref(n)), "tl3_serialize")
+        _check(fn(self._h, None, ctypes.byref(n)), "tl3_serialize")
         buf = ctypes.create_string_buffer(n.value)
-        _check(lib().tl3_serialize(self._h, buf, ctypes.byref(n)), "tl3_serialize")
+        _check(fn(self._h, buf, ctypes.byref(n)), "tl3_serialize")
         return buf.raw[:n.value]
 
     # -- device side -------------------------------------------------------------------------

@@ -494,3 +494,62 @@ print("rank", rank, "ok")
     for rank, (p, out) in enumerate(zip(procs, outs)):
         assert p.returncode == 0, out
         assert f"rank {rank} ok" in out
+
+
+@pytest.mark.parametrize("sparsity,tiles", [(0.3, (128, 128)), (0.5, (128, 128)), (0.7, (128, 128)), (0.6, (4, 32)), (0.95, (128, 128))])
+def test_compact_persistence_round_trip(tl3, sparsity, tiles):
+    """tl3_serialize_compact -> tl3_deserialize gives the same container: re-serialised in the plain
+    form it is the original's plain bytes.  Its size is the header, thirteen lengths and what
+    tl3_stats announces; above and below 50 % it is smaller than the plain form."""
+    W = wl.Case(0, "cp", 300, 520, 8, 33, sparsity, "magnitude").make_W()
+    W[5, 7] = np.float16(-0.0)                                     # a zero as far as the format is concerned
+    m = tl3.encode(W, tile_m=tiles[0], tile_k=tiles[1])
+    plain, compact = m.serialize(), m.serialize(compact=True)
+    back = tl3.Matrix.deserialize(compact)
+    assert back.serialize() == plain
+    assert back.serialize(compact=True) == compact
+    assert np.array_equal(back.decode(), m.decode())
+    header = len(plain) - 9 * 8 - m.stats()["canonical_bytes"]
+    assert len(compact) == header + 13 * 8 + m.stats()["canonical_bytes_compact_all"]
+    if sparsity != 0.5:
+        assert len(compact) < len(plain)
+
+
+def test_corrupted_compact_containers_are_rejected_or_valid(tl3):
+    """Nothing in a compact container is trusted: truncations, and single bytes overwritten anywhere
+    in the directories, bitmaps, lists and values, either fail with BAD_CONTAINER or give a container
+    that serialises again and decodes or is refused by the decoder; none may crash or read out of
+    bounds."""
+    rng = np.random.default_rng(17)
+    W = wl.Case(0, "cc", 260, 300, 8, 5, 0.4, "magnitude").make_W()
+    W[128:, :] = np.where(rng.random((132, 300)) < 0.25, W[128:, :], np.float16(0))      # sparse lower half: bitmap tiles
+    m = tl3.encode(W)
+    good = m.serialize(compact=True)
+    assert tl3.Matrix.deserialize(good).serialize() == m.serialize()
+    modes_v, modes_r = m.canonical("val_dir").reshape(-1, 2)[:, 0], m.canonical("res_dir").reshape(-1, 2)[:, 0]
+    assert set(modes_v.tolist()) == {0, 1} and set(modes_r.tolist()) == {0, 1}           # both forms of both layers occur
+    for cut in (0, 50, 79, 80, 200, len(good) // 2, len(good) - 1):
+        with pytest.raises(tl3.Tl3Error):
+            tl3.Matrix.deserialize(good[:cut])
+    with pytest.raises(tl3.Tl3Error):
+        tl3.Matrix.deserialize(good + b"\0")
+    rejected = accepted = 0
+    # the first kilobyte holds the header and the value directory; then spread over the whole blob
+    places = list(range(40, 400)) + rng.integers(0, len(good), size=600).tolist()
+    for at in places:
+        bad = bytearray(good)
+        bad[at] ^= int(rng.integers(1, 256))
+        try:
+            back = tl3.Matrix.deserialize(bytes(bad))
+        except tl3.Tl3Error as e:
+            assert e.code == tl3.ERR_BAD_CONTAINER
+            rejected += 1
+            continue
+        accepted += 1                                             # e.g. a changed value: still a container
+        assert len(back.serialize()) > 0
+        try:
+            assert back.decode().shape == W.shape
+        except tl3.Tl3Error as e:                                 # the decoder walks the chains and may still refuse
+            assert e.code == tl3.ERR_BAD_CONTAINER
+        back.close()
+    assert rejected > 100 and accepted > 100
