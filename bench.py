@@ -221,8 +221,9 @@ class Weights:
         # the same container built by the CUDA encoder (window classification, scans, pairing, chain
         # emission on the GPU; the copy of the arrays back to the host is inside the time)
         self.device_encode_s, self.device_encode_identical, self.device_pack_s, self.device_pack_identical = None, None, None, None
+        self.device_convert_s, self.device_convert_identical = None, None
         if dense:
-            enc, pack = [], []
+            enc, pack, conv = [], [], []
             for _ in range(2):                               # best of two: the first call of a kind pays for the module load
                 t0 = time.perf_counter()
                 md = tl3.Matrix.encode_on_device(self.dense[0])
@@ -238,7 +239,17 @@ class Weights:
                 self.device_pack_identical = bool(torch.equal(blob_d, first))
                 del blob_d
                 md.close()
-            self.device_encode_s, self.device_pack_s = min(enc), min(pack)
+                # ... and the whole conversion without a host copy of the container: dense W on the
+                # device -> packed blob on the device (encode, layout pass, blob pass)
+                t0 = time.perf_counter()
+                mo = tl3.Matrix.encode_on_device(self.dense[0], device_only=True)
+                blob_o = mo.upload_packed_on_device(device=dev)
+                torch.cuda.synchronize()
+                conv.append(time.perf_counter() - t0)
+                self.device_convert_identical = bool(torch.equal(blob_o, first))
+                del blob_o
+                mo.close()
+            self.device_encode_s, self.device_pack_s, self.device_convert_s = min(enc), min(pack), min(conv)
 
     def spmm(self, i, X, Y, ws, stream=None):
         self.m.bind(self.blobs[i % len(self.blobs)])
@@ -305,6 +316,7 @@ def run_ours(args, rank, local_rank, world):
         conversion.append({"M": c.M, "K": c.K, "host_encode_s": round(wt.encode_s, 3), "device_pack_upload_s": round(wt.upload_s, 3),
                            "gpu_encode_s": round(wt.device_encode_s, 3), "gpu_encode_identical": wt.device_encode_identical,
                            "gpu_pack_s": round(wt.device_pack_s, 3), "gpu_pack_identical": wt.device_pack_identical,
+                           "gpu_convert_on_device_s": round(wt.device_convert_s, 4), "gpu_convert_identical": wt.device_convert_identical,
                            "canonical_bytes": st["canonical_bytes"], "device_bytes": st["device_bytes"],
                            # shares of the non-zeros by layer: the canonical container, and the device image that
                            # actually streams (its chains are cut after three code words, the tails travel as

@@ -115,6 +115,14 @@ int tl3_encode(const uint16_t* W, int64_t M, int64_t K, const tl3_params* params
  *   of the container (cudaMalloc), runs on `stream` and waits for it.
  * Errors: INVALID_ARG, UNSUPPORTED (more than 4 GiB of PDD bytes), CUDA, NO_MEMORY. */
 int tl3_encode_device(const void* dW, int64_t M, int64_t K, int64_t ldw, void* stream, tl3_matrix** out);
+/* The same conversion for a matrix that is only going to be multiplied: the container stays on the
+ * device, no host copy of it is made, and the handle comes back planned (tl3_device_bytes() is
+ * valid).  tl3_upload_device() then packs it into the caller's blob and releases the device copy
+ * of the container; tl3_spmm*, tl3_bind, tl3_stats (layer counts; the sizes of the compact forms
+ * read -1), tl3_workspace_bytes and tl3_free work as on any handle.  The calls that need the
+ * container on the host -- tl3_decode, tl3_canonical, tl3_serialize*, tl3_pack, tl3_upload --
+ * return UNSUPPORTED.  dW, ldw, stream, errors: as for tl3_encode_device. */
+int tl3_encode_device_only(const void* dW, int64_t M, int64_t K, int64_t ldw, void* stream, tl3_matrix** out);
 
 /* Decode back to dense: Algorithm 1 run on the host, then the 2:4 expansion and the Residual
  * entries.  W_out: host, M*K uint16_t, caller-owned, fully overwritten.  The result equals the

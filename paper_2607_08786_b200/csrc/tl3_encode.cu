@@ -308,7 +308,22 @@ tl3_encode_scan_kernel(uint32_t* tile_dir, long long n_tiles, unsigned long long
 }  // namespace
 }  // namespace tl3
 
-extern "C" int tl3_encode_device(const void* dW, int64_t M, int64_t K, int64_t ldw, void* stream, tl3_matrix** out) {
+namespace tl3 {
+namespace {
+void release_encoded(void* p) {
+  DeviceCanon* c = static_cast<DeviceCanon*>(p);
+  if (!c) return;
+  for (void* a : c->alloc) if (a) cudaFree(a);
+  delete c;
+}
+}  // namespace
+}  // namespace tl3
+
+extern "C" int tl3_plan_device(tl3_matrix* m, void* stream);
+
+// keep_on_device: leave the container where the kernels wrote it (for tl3_upload_device) and make
+// no host copies of it.
+static int encode_device_impl(const void* dW, int64_t M, int64_t K, int64_t ldw, void* stream, bool keep_on_device, tl3_matrix** out) {
   using namespace tl3;
   if (!dW || !out || M <= 0 || K <= 0 || ldw < K || M > (int64_t{1} << 31) || K > (int64_t{1} << 31)) return TL3_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -360,6 +375,22 @@ extern "C" int tl3_encode_device(const void* dW, int64_t M, int64_t K, int64_t l
     a.emit = 1;
     tl3_encode_kernel<<<static_cast<unsigned>(m->n_tiles), kEncThreads, 0, st>>>(a);
     TL3_ENC_CUDA(cudaGetLastError());
+    if (keep_on_device) {
+      TL3_ENC_CUDA(cudaMemcpyAsync(stats, a.stats, sizeof(stats), cudaMemcpyDeviceToHost, st));
+      TL3_ENC_CUDA(cudaStreamSynchronize(st));
+      m->nnz = static_cast<int64_t>(stats[0]); m->n_tc = static_cast<int64_t>(stats[1]); m->n_sf = static_cast<int64_t>(stats[2]);
+      m->n_res = static_cast<int64_t>(stats[3]); m->n_dummy = static_cast<int64_t>(stats[4]); m->n_slots_unused = static_cast<int64_t>(stats[5]);
+      DeviceCanon* c = new (std::nothrow) DeviceCanon();
+      if (!c) { rc = TL3_ERR_NO_MEMORY; goto done; }
+      *c = DeviceCanon{a.tc_vals, a.tc_meta, a.chain_tau0, a.chain_rho0, a.chain_len, a.pdd_bytes, a.tile_dir, a.res_rho, a.res_val, {scratch, var}};
+      m->device_canon = c;
+      m->release_device_canon = release_encoded;
+      m->host_arrays = false;
+      m->canon_bytes = static_cast<int64_t>(n_vals * 2 + n_meta + n_chain * 5 + n_dir * 4 + totals[0] + totals[1] * 4);
+      scratch = nullptr;                                            // owned by the handle from here on
+      var = nullptr;
+      goto done;
+    }
     try {
       m->tc_vals.resize(n_vals); m->tc_meta.resize(n_meta);
       m->chain_tau0.resize(n_chain); m->chain_rho0.resize(n_chain); m->chain_len.resize(n_chain);
@@ -385,7 +416,16 @@ extern "C" int tl3_encode_device(const void* dW, int64_t M, int64_t K, int64_t l
 done:
   if (scratch) cudaFree(scratch);
   if (var) cudaFree(var);
-  if (rc != TL3_OK) { delete m; return rc; }
+  if (rc == TL3_OK && keep_on_device) rc = tl3_plan_device(m, stream);   // sizes of the packed blocks: tl3_device_bytes() is valid on return
+  if (rc != TL3_OK) { tl3_free(m); return rc; }
   *out = m;
   return TL3_OK;
+}
+
+extern "C" int tl3_encode_device(const void* dW, int64_t M, int64_t K, int64_t ldw, void* stream, tl3_matrix** out) {
+  return encode_device_impl(dW, M, K, ldw, stream, false, out);
+}
+
+extern "C" int tl3_encode_device_only(const void* dW, int64_t M, int64_t K, int64_t ldw, void* stream, tl3_matrix** out) {
+  return encode_device_impl(dW, M, K, ldw, stream, true, out);
 }

@@ -303,6 +303,7 @@ int tl3_encode(const uint16_t* W, int64_t M, int64_t K, const tl3_params* params
 
 int tl3_decode(const tl3_matrix* m, uint16_t* W_out) {
   if (!m || !W_out) return TL3_ERR_INVALID_ARG;
+  if (!m->host_arrays) return TL3_ERR_UNSUPPORTED;               // tl3_encode_device_only: the container is not on the host
   if (!consistent(*m)) return TL3_ERR_BAD_CONTAINER;
   const int TM = m->p.tile_m, TK = m->p.tile_k, H = TK / 2;
   const int64_t half_ld = m->K_pad / 2, meta_ld = m->K_pad / 8;
@@ -436,6 +437,7 @@ static void ensure_val_compact(const tl3_matrix* m) {
 
 int tl3_canonical(const tl3_matrix* m, int which, const void** ptr, size_t* bytes) {
   if (!m || !ptr || !bytes) return TL3_ERR_INVALID_ARG;
+  if (!m->host_arrays) return TL3_ERR_UNSUPPORTED;
   if (which >= TL3_RES_DIR && which <= TL3_RES_MASK) ensure_compact(m);
   if (which >= TL3_VAL_DIR && which <= TL3_VAL_MASK) ensure_val_compact(m);
   switch (which) {
@@ -470,8 +472,15 @@ int tl3_stats(const tl3_matrix* m, tl3_stats_t* out) {
   out->M = m->M; out->K = m->K; out->M_pad = m->M_pad; out->K_pad = m->K_pad; out->n_tiles = m->n_tiles;
   out->nnz = m->nnz; out->n_tc = m->n_tc; out->n_sf = m->n_sf; out->n_res = m->n_res;
   out->n_dummy = m->n_dummy; out->n_slots_unused = m->n_slots_unused;
-  out->canonical_bytes = canonical_bytes(m);
   out->device_bytes = static_cast<int64_t>(tl3_device_bytes(m));
+  out->dev_n_sf = m->dev_n_sf; out->dev_n_res = m->dev_n_res; out->dev_n_dummy = m->dev_n_dummy;
+  out->dev_pdd_bytes = m->dev_pdd_bytes;
+  if (!m->host_arrays) {                                           // the sizes of the compact forms need the arrays
+    out->canonical_bytes = m->canon_bytes;
+    out->canonical_bytes_compact = out->canonical_bytes_compact_all = -1;
+    return TL3_OK;
+  }
+  out->canonical_bytes = canonical_bytes(m);
   ensure_compact(m);
   out->canonical_bytes_compact = out->canonical_bytes - static_cast<int64_t>(m->res_rho.size() * 2) +
                                  static_cast<int64_t>(m->res_dir.size() * 4 + m->res_list.size() * 2 + m->res_mask.size());
@@ -496,6 +505,7 @@ struct FileHeader {
 
 int tl3_serialize(const tl3_matrix* m, void* buf, size_t* bytes) {
   if (!m || !bytes) return TL3_ERR_INVALID_ARG;
+  if (!m->host_arrays) return TL3_ERR_UNSUPPORTED;
   size_t need = sizeof(FileHeader);
   for (int w = 0; w < 9; ++w) {
     const void* p; size_t n;
@@ -528,6 +538,7 @@ static const int kCompactOrder[13] = {TL3_VAL_DIR, TL3_VAL_PACK, TL3_VAL_MASK, T
 
 int tl3_serialize_compact(const tl3_matrix* m, void* buf, size_t* bytes) {
   if (!m || !bytes) return TL3_ERR_INVALID_ARG;
+  if (!m->host_arrays) return TL3_ERR_UNSUPPORTED;
   size_t need = sizeof(FileHeader);
   for (int w : kCompactOrder) {
     const void* p; size_t n;

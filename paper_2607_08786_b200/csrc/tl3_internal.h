@@ -29,8 +29,13 @@ struct tl3_matrix {
   void* dptr = nullptr;
   // device copies of the canonical arrays between tl3_plan_device and tl3_upload_device (one
   // cudaMalloc, released by tl3_upload_device or tl3_free through `release_device_canon`)
-  void* device_canon = nullptr;
+  void* device_canon = nullptr;             // a tl3::DeviceCanon
   void (*release_device_canon)(void*) = nullptr;
+  // false for a handle made by tl3_encode_device_only: the nine arrays above are empty, the
+  // container lives on the device until tl3_upload_device has packed it, and `canon_bytes` keeps
+  // the sizes the arrays would have
+  bool host_arrays = true;
+  int64_t canon_bytes = 0;
   // Layout of the device image, computed on first use (tl3_device_bytes, tl3_pack, tl3_upload,
   // tl3_stats) under `layout_mu`, so that calls that take a const handle may share it between
   // threads; `layout_ready` is set last.
@@ -57,6 +62,13 @@ struct tl3_matrix {
 };
 
 namespace tl3 {
+
+// The canonical arrays on the device (between an encode or a copy there and tl3_upload_device).
+struct DeviceCanon {
+  const uint16_t* tc_vals; const uint8_t* tc_meta; const uint16_t* chain_tau0; const uint16_t* chain_rho0;
+  const uint8_t* chain_len; const uint8_t* pdd_bytes; const uint32_t* tile_dir; const uint16_t* res_rho; const uint16_t* res_val;
+  void* alloc[2];                            // what to cudaFree
+};
 
 // ---- device blob layout ------------------------------------------------------------------
 // [0, 256)                 header (magic, shape; informational)

@@ -334,7 +334,12 @@ struct CanonOnDevice {
   PackArgs args{};
 };
 
-void release_canon(void* p) { cudaFree(p); }
+void release_canon(void* p) {
+  DeviceCanon* c = static_cast<DeviceCanon*>(p);
+  if (!c) return;
+  for (void* a : c->alloc) if (a) cudaFree(a);
+  delete c;
+}
 
 #define TL3_PK_CUDA(expr)                                     \
   do {                                                        \
@@ -357,24 +362,31 @@ int canon_to_device(tl3_matrix* m, cudaStream_t st, PackArgs* out) {
   off[0] = 0;
   for (int i = 0; i < 9; ++i) off[i + 1] = off[i] + up(sz[i] + 16);
   if (!m->device_canon) {
+    if (!m->host_arrays) return TL3_ERR_UNSUPPORTED;           // a device-only handle whose container has been packed and released
     void* p = nullptr;
     TL3_PK_CUDA(cudaMalloc(&p, off[9]));
-    m->device_canon = p;
+    DeviceCanon* c = new (std::nothrow) DeviceCanon();
+    if (!c) { cudaFree(p); return TL3_ERR_NO_MEMORY; }
+    uint8_t* b = static_cast<uint8_t*>(p);
+    *c = DeviceCanon{reinterpret_cast<const uint16_t*>(b + off[0]), b + off[1], reinterpret_cast<const uint16_t*>(b + off[2]),
+                     reinterpret_cast<const uint16_t*>(b + off[3]), b + off[4], b + off[5], reinterpret_cast<const uint32_t*>(b + off[6]),
+                     reinterpret_cast<const uint16_t*>(b + off[7]), reinterpret_cast<const uint16_t*>(b + off[8]), {p, nullptr}};
+    m->device_canon = c;
     m->release_device_canon = release_canon;
     for (int i = 0; i < 9; ++i)
-      if (sz[i]) TL3_PK_CUDA(cudaMemcpyAsync(static_cast<uint8_t*>(p) + off[i], src[i], sz[i], cudaMemcpyHostToDevice, st));
+      if (sz[i]) TL3_PK_CUDA(cudaMemcpyAsync(b + off[i], src[i], sz[i], cudaMemcpyHostToDevice, st));
   }
-  uint8_t* b = static_cast<uint8_t*>(m->device_canon);
+  const DeviceCanon* c = static_cast<const DeviceCanon*>(m->device_canon);
   PackArgs a{};
-  a.tc_vals = reinterpret_cast<const uint16_t*>(b + off[0]);
-  a.tc_meta = b + off[1];
-  a.chain_tau0 = reinterpret_cast<const uint16_t*>(b + off[2]);
-  a.chain_rho0 = reinterpret_cast<const uint16_t*>(b + off[3]);
-  a.chain_len = b + off[4];
-  a.pdd_bytes = b + off[5];
-  a.tile_dir = reinterpret_cast<const uint32_t*>(b + off[6]);
-  a.res_rho = reinterpret_cast<const uint16_t*>(b + off[7]);
-  a.res_val = reinterpret_cast<const uint16_t*>(b + off[8]);
+  a.tc_vals = c->tc_vals;
+  a.tc_meta = c->tc_meta;
+  a.chain_tau0 = c->chain_tau0;
+  a.chain_rho0 = c->chain_rho0;
+  a.chain_len = c->chain_len;
+  a.pdd_bytes = c->pdd_bytes;
+  a.tile_dir = c->tile_dir;
+  a.res_rho = c->res_rho;
+  a.res_val = c->res_val;
   a.K_pad = m->K_pad;
   a.tiles_k = static_cast<int>(m->tiles_k);
   *out = a;
@@ -448,7 +460,7 @@ extern "C" int tl3_upload_device(tl3_matrix* m, void* dptr, void* stream) {
   }
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);          // header, offsets and the canonical copies are released below
   cudaFree(d_off);
-  if (m->device_canon) { cudaFree(m->device_canon); m->device_canon = nullptr; }
+  if (m->device_canon) { release_canon(m->device_canon); m->device_canon = nullptr; }
   if (e != cudaSuccess) { set_cuda_error(static_cast<int>(e)); return TL3_ERR_CUDA; }
   m->dptr = dptr;
   return TL3_OK;

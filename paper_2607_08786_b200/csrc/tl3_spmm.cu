@@ -994,6 +994,7 @@ size_t tl3_device_bytes(const tl3_matrix* m) {
 
 int tl3_pack(const tl3_matrix* m, void* host_buf, size_t bytes) {
   if (!m || !host_buf) return TL3_ERR_INVALID_ARG;
+  if (!m->host_arrays) return TL3_ERR_UNSUPPORTED;               // tl3_encode_device_only: pack with tl3_upload_device
   if (m->p.tile_m != tl3::kTileM || m->p.tile_k != tl3::kTileK) return TL3_ERR_UNSUPPORTED;
   if (bytes < tl3::plan_device_layout(m)) return TL3_ERR_INVALID_ARG;
   tl3::pack_device_blob(m, static_cast<uint8_t*>(host_buf));
@@ -1003,6 +1004,7 @@ int tl3_pack(const tl3_matrix* m, void* host_buf, size_t bytes) {
 int tl3_upload(tl3_matrix* m, void* dptr, void* stream) {
   if (!m || !dptr || (reinterpret_cast<uintptr_t>(dptr) & 255) != 0) return TL3_ERR_INVALID_ARG;
   if (m->p.tile_m != tl3::kTileM || m->p.tile_k != tl3::kTileK) return TL3_ERR_UNSUPPORTED;
+  if (!m->host_arrays) return TL3_ERR_UNSUPPORTED;               // tl3_encode_device_only: pack with tl3_upload_device
   const size_t bytes = tl3::plan_device_layout(m);
   std::vector<uint8_t> staging;
   try {

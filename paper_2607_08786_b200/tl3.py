@@ -29,7 +29,7 @@ _CANONICAL_DTYPES = (np.uint16, np.uint8, np.uint16, np.uint16, np.uint8, np.uin
                      np.uint16, np.uint16, np.uint32, np.uint16, np.uint8, np.uint32, np.uint16, np.uint8)
 
 # every symbol include/tl3.h declares
-SYMBOLS = ("tl3_encode", "tl3_encode_device", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_serialize_compact", "tl3_deserialize",
+SYMBOLS = ("tl3_encode", "tl3_encode_device", "tl3_encode_device_only", "tl3_decode", "tl3_canonical", "tl3_stats", "tl3_serialize", "tl3_serialize_compact", "tl3_deserialize",
            "tl3_free", "tl3_device_bytes", "tl3_pack", "tl3_upload", "tl3_bind", "tl3_plan_device", "tl3_upload_device", "tl3_workspace_bytes", "tl3_workspace_init",
            "tl3_spmm", "tl3_spmm_ex", "tl3_spmm_nt", "tl3_spmm_host", "tl3_spmm_host_async", "tl3_spmm_static_scratch", "tl3_static_scratch_status", "tl3_status", "tl3_status_word", "tl3_selftest_bounded_wait", "tl3_last_launch", "tl3_strerror",
            "tl3_last_cuda_error", "tl3_get_tuning", "tl3_set_tuning")
@@ -83,6 +83,7 @@ def lib() -> ctypes.CDLL:
         vp, i64, sz, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_int
         L.tl3_encode.argtypes = [vp, i64, i64, ctypes.POINTER(Params), ctypes.POINTER(vp)]
         L.tl3_encode_device.argtypes = [vp, i64, i64, i64, vp, ctypes.POINTER(vp)]
+        L.tl3_encode_device_only.argtypes = [vp, i64, i64, i64, vp, ctypes.POINTER(vp)]
         L.tl3_decode.argtypes = [vp, vp]
         L.tl3_canonical.argtypes = [vp, ci, ctypes.POINTER(vp), ctypes.POINTER(sz)]
         L.tl3_stats.argtypes = [vp, ctypes.POINTER(Stats)]
@@ -167,14 +168,15 @@ class Matrix:
         return cls(h.value)
 
     @classmethod
-    def encode_on_device(cls, W, stream=None) -> "Matrix":
-        """The same container, built by the GPU encoder from a torch.float16 matrix on the device."""
+    def encode_on_device(cls, W, stream=None, device_only: bool = False) -> "Matrix":
+        """The same container, built by the GPU encoder from a torch.float16 matrix on the device.
+        ``device_only=True`` keeps it there (no host copy): follow with ``upload_packed_on_device``."""
         import torch
         if W.dtype != torch.float16 or W.dim() != 2 or W.stride(1) != 1 or not W.is_cuda:
             raise ValueError("W must be a 2-D float16 CUDA tensor with contiguous rows")
         h = ctypes.c_void_p()
-        _check(lib().tl3_encode_device(W.data_ptr(), W.shape[0], W.shape[1], W.stride(0), _stream_ptr(stream), ctypes.byref(h)),
-               "tl3_encode_device")
+        fn = lib().tl3_encode_device_only if device_only else lib().tl3_encode_device
+        _check(fn(W.data_ptr(), W.shape[0], W.shape[1], W.stride(0), _stream_ptr(stream), ctypes.byref(h)), "tl3_encode_device")
         return cls(h.value)
 
     @classmethod

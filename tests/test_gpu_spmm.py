@@ -806,3 +806,51 @@ def test_random_shapes_through_every_gpu_route(tl3, oracle_mod):
         assert np.all(np.abs(Yb - want) <= oracle_mod.tolerance(bound + np.abs(bias.astype(np.float64))[:, None])), tag
         m.close()
         ref.close()
+
+
+@pytest.mark.parametrize("shape,sparsity,kind", [((1024, 1024), 0.5, "bernoulli"), ((640, 896), 0.4, "magnitude"),
+                                                 ((1000, 1096), 0.6, "magnitude"), ((130, 260), 0.9, "magnitude"),
+                                                 ((2048, 4096), 0.5, "wanda")])
+def test_conversion_that_never_leaves_the_gpu(tl3, oracle_mod, shape, sparsity, kind):
+    """Dense W on the device -> container on the device -> packed blob on the device, with no host
+    copy of the container: the blob must be the host pipeline's blob byte for byte, the layer counts
+    the host encoder's, the product right, and every call that needs the container on the host must
+    say so instead of handing out empty arrays."""
+    import torch
+    case = wl.Case(0, "dev_only", shape[0], shape[1], 16, 130 + shape[0], sparsity, kind)
+    W, X = case.make_W(), case.make_X()
+    ref = tl3.encode(W)
+    want = ref.pack()
+    m = tl3.Matrix.encode_on_device(torch.from_numpy(W).cuda(), device_only=True)
+    assert m.device_bytes() == want.size
+    blob = m.upload_packed_on_device()
+    torch.cuda.synchronize()
+    assert np.array_equal(blob.cpu().numpy(), want)
+    st, st_ref = m.stats(), ref.stats()
+    for key in st:
+        if key.startswith("canonical_bytes_compact"):
+            assert st[key] == -1
+        else:
+            assert st[key] == st_ref[key], key
+    Y = m.spmm(device_X(X))
+    torch.cuda.synchronize()
+    check(oracle_mod, W, X, Y.cpu().numpy(), with_oracle_spmm=False)
+    for call in (m.decode, lambda: m.canonical("tc_vals"), m.serialize, lambda: m.serialize(compact=True), m.pack, m.upload):
+        with pytest.raises(tl3.Tl3Error) as e:
+            call()
+        assert e.value.code == tl3.ERR_UNSUPPORTED
+    with pytest.raises(tl3.Tl3Error):                             # the device copy of the container is gone after packing
+        m.upload_packed_on_device()
+    m.close()
+    # a handle that is freed before it was packed releases its device memory (checked where the
+    # container is large enough to tell from allocator noise)
+    if W.nbytes >= (8 << 20):
+        Wd = torch.from_numpy(W).cuda()
+        torch.cuda.synchronize()
+        free0 = torch.cuda.mem_get_info()[0]
+        m2 = tl3.Matrix.encode_on_device(Wd, device_only=True)
+        held = free0 - torch.cuda.mem_get_info()[0]
+        assert held >= W.nbytes // 2                              # the container is on the device now
+        m2.close()
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] >= free0 - (2 << 20)
