@@ -55,7 +55,8 @@ def test_static_scratch_entry_point_matches_the_regular_one(oracle_mod):
     rc = L.tl3_spmm_static_scratch(m._h, Xd.data_ptr(), Xd.stride(0), Y.data_ptr(), Y.stride(0), case.N, stream)
     assert rc == tl3.OK
     torch.cuda.synchronize()
-    assert torch.cuda.mem_get_info()[0] == free_before and torch.cuda.memory_allocated() == booked_before
+    # (>=: memory that an earlier test handed back may still be on its way to the free pool)
+    assert torch.cuda.mem_get_info()[0] >= free_before and torch.cuda.memory_allocated() == booked_before
 
 
 def test_static_scratch_refuses_what_does_not_fit():
